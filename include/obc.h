@@ -1,0 +1,150 @@
+/*
+ * obc.h -- C ABI of the B200 (sm_100a) ExactOBS / OBQ layer solver ("Optimal Brain Compression").
+ *
+ * One layer is a weight matrix W (d_row x d_col) and calibration inputs X (d_col x N), as in the paper's
+ * layer-wise compression problem (Section 2, Eq. 2).  The calls below are the stages of the method:
+ *
+ *   obc_hessian            H = 2 X X^T, accumulated over chunks of N          (Section 3, "ExactOBS")
+ *   obc_hessian_inverse    Hinv = inv(H + damp I)                             (Section 3, "Implementation Details")
+ *   obc_prune_trace        Algorithm 1 on every row: order P, loss trace L    (Section 3, Steps 1-2)
+ *   obc_select_global_mask Algorithm 2: global mask with k pruned weights     (appendix, global step)
+ *   obc_prune_apply        remaining weights for the chosen per-row counts    (Section 3, Figure 1)
+ *   obc_minmax_grid        per-row uniform grid over the kept weights
+ *   obc_quantize           Algorithm 3 (OBQ), optionally after a pruning replay (Section 4; Section 6 setup)
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The library
+ *     allocates nothing, frees nothing and keeps no state between calls.  Scratch memory comes from the
+ *     caller's workspace `ws` of at least obc_workspace_bytes(...) bytes (256-byte aligned).
+ *   - Matrices are row-major FP32 with a leading dimension in elements.  Base pointers of FP32 matrices
+ *     are 16-byte aligned and leading dimensions are multiples of 4.
+ *   - Calls enqueue work on `stream` and return without synchronising.  Argument errors are found on the
+ *     host and returned before anything is launched or written.  Data-dependent failures never trap: they
+ *     are written to `info` / `row_status` in device memory.
+ *   - row_begin / row_count select a row range; outputs of other rows are not touched, so a layer can be
+ *     split across calls (or devices) and resumed by range.
+ *   - Original column indices are 0-based.  mask: 1 = kept, 0 = pruned.
+ */
+#ifndef OBC_H_
+#define OBC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OBC_OK = 0,
+    OBC_ERR_INVALID_ARG = 1,   /* NULL pointer, negative or inconsistent size, unknown enum              */
+    OBC_ERR_ALIGNMENT = 2,     /* pointer not 16-byte aligned or leading dimension not a multiple of 4   */
+    OBC_ERR_WORKSPACE = 3,     /* ws is NULL, misaligned or smaller than obc_workspace_bytes(...)        */
+    OBC_ERR_NOT_POSDEF = 4,    /* (reported through info[]) Cholesky met a non-positive pivot            */
+    OBC_ERR_NONFINITE = 5,     /* (reported through row_status[]) non-positive / non-finite [Hinv]_pp    */
+    OBC_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired                                     */
+    OBC_ERR_CUDA = 7,          /* a CUDA runtime call failed (launch configuration, missing device ...)  */
+    OBC_ERR_UNSUPPORTED = 8    /* size outside what the kernels support (d_col > OBC_MAX_DCOL)           */
+} obc_status;
+
+typedef enum { OBC_PREC_FP32 = 0, OBC_PREC_TF32 = 1, OBC_PREC_BF16X3 = 2 } obc_prec;
+
+enum {
+    OBC_FLAG_OUTLIERS = 1      /* obc_quantize: quantise weights whose error exceeds Delta/2 first
+                                  (Section 4, "Quantization Outliers"); off = plain argmin of Eq. 7      */
+};
+
+typedef enum {
+    OBC_OP_HESSIAN = 0, OBC_OP_INVERSE = 1, OBC_OP_PRUNE_TRACE = 2, OBC_OP_SELECT = 3,
+    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5
+} obc_op;
+
+#define OBC_MAX_DCOL 5120      /* per-row state of the elimination engine lives in one CTA's shared memory */
+
+typedef void *obc_stream;      /* a cudaStream_t (NULL = default stream) */
+
+const char *obc_status_string(obc_status s);
+
+/* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).
+ * n is only used by OBC_OP_HESSIAN; row_count (the rows one call processes) by the three row-engine ops,
+ * where 0 means "size for any row_count".  Returns 0 on invalid arguments. */
+size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n);
+
+/* Section 3 ("ExactOBS"): the Hessian of every row's least-squares problem is H = 2 X X^T.
+ * X: d_col x n, row-major, ldx >= n (one chunk of the calibration axis).  H: d_col x d_col, ldh >= d_col.
+ * accumulate = 0 overwrites H, 1 adds to it (Section 3, "Implementation Details": further samples are
+ * accumulated into the Hessian once).  H is written in full (both triangles, exactly symmetric).
+ * prec picks the tensor-core input precision of the contraction; accumulation is FP32. */
+obc_status obc_hessian(const float *X, int d_col, int64_t n, int64_t ldx,
+                       float *H, int ldh, int accumulate, obc_prec prec,
+                       void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Section 3 ("Implementation Details"): Hinv = inv(H + damp_rel * mean(diag H) * I) through a Cholesky
+ * factorisation carried in FP64, written as an exactly symmetric FP32 matrix (ldhi >= d_col).
+ * info[0] (device int32) = 0, or 1 + index of the first non-positive pivot (Hinv is then undefined). */
+obc_status obc_hessian_inverse(const float *H, int d_col, int ldh, float damp_rel,
+                               float *Hinv, int ldhi, int32_t *info,
+                               void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Algorithm 1 for rows [row_begin, row_begin+row_count) of W (d_row x d_col, ldw >= d_col), each on its
+ * own FP32 copy of Hinv: `steps` (1..d_col) greedy eliminations; step t removes
+ * p = argmin_{p in M} w_p^2 / [Hinv]_pp (ties: lowest index), compensates the remaining weights (Eq. 3)
+ * and eliminates p from the row's inverse Hessian (Lemma 1).
+ *   order  : d_row x d_col int32, order[r][t] = column removed at step t        (entries t >= steps untouched)
+ *   loss   : d_row x d_col FP32,  loss[r][t] = w_p^2/[Hinv]_pp at that moment   (Section 3, Step 2)
+ *   w_trace: NULL, or d_row x (steps+1) x d_col FP32: the whole row after t = 0..steps eliminations
+ *            (Figure 1, the "more memory" option)
+ *   row_status: d_row int32, 0 or 1+t if [Hinv]_pp was non-positive / non-finite at step t (the row stops:
+ *            its later order entries are -1 and loss entries +inf). */
+obc_status obc_prune_trace(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                           const float *Hinv, int ldhi, int steps,
+                           int32_t *order, float *loss, float *w_trace, int32_t *row_status,
+                           void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Algorithm 2 (appendix, "ExactOBS Global Step"): repeatedly prune, across all rows, the weight whose
+ * next recorded loss is smallest (ties: lowest row), k times.  k is a count, 0 <= k <= d_row*d_col.
+ *   counts: d_row int32, weights pruned per row;  mask: d_row x d_col uint8, 0 at order[r][t], t < counts[r].
+ * The result is exactly the sequential procedure's (computed as a selection over prefix-maximum keys). */
+obc_status obc_select_global_mask(const float *loss, const int32_t *order, int d_row, int d_col, int64_t k,
+                                  int32_t *counts, uint8_t *mask,
+                                  void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Section 3 / Figure 1: the weights of each row after its first counts[r] eliminations.
+ * w_trace != NULL (layout of obc_prune_trace with this `trace_steps`): rows are gathered from the trace.
+ * w_trace == NULL: the eliminations order[r][0..counts[r]) are replayed on W (no argmin). */
+obc_status obc_prune_apply(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                           const float *Hinv, int ldhi, const int32_t *order, const int32_t *counts,
+                           const float *w_trace, int trace_steps,
+                           float *W_out, int ldwo, int32_t *row_status,
+                           void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Per-row uniform grid over the kept entries (mask NULL = all kept); the range always contains 0.
+ *   asymmetric: maxq = 2^bits-1, scale = (hi-lo)/maxq, zero = rne(-lo/scale)
+ *   symmetric : Q = 2^(bits-1)-1, scale = max|w|/Q, zero = Q, maxq = 2Q
+ * A row without spread gets scale = 1.  bits in 2..16.  *maxq_host (host pointer, nullable) receives maxq.
+ * The paper fixes only "symmetric / asymmetric per-channel grids" (Section 6); this min-max rule is the
+ * benchmark configurations' choice, and any other grid can be passed to obc_quantize instead. */
+obc_status obc_minmax_grid(const float *W, int ldw, int d_row, int d_col, const uint8_t *mask,
+                           int bits, int symmetric, float *scale, float *zero, int *maxq_host,
+                           obc_stream stream);
+
+/* Algorithm 3 (OBQ) for a row range: like Algorithm 1 with the target q(w_p) instead of 0 (Eq. 7), where
+ * q(x) = scale * (clamp(rne(x/scale) + zero, 0, maxq) - zero) and maxq follows from bits/symmetric as above.
+ *   prune_order / prune_counts == NULL: scale, zero (d_row FP32) are INPUTS; all d_col weights are quantised.
+ *   otherwise (compound, Section 6 "Experimental Setup": sparsify first, then quantise the rest): the first
+ *     prune_counts[r] eliminations of prune_order[r] are replayed, the row's min-max grid is built from the
+ *     compensated survivors and written to scale/zero (OUTPUTS), and only the survivors are quantised.
+ *   W_out  : d_row x d_col FP32 (ldwo), quantised weights (pruned entries 0)
+ *   codes  : d_row x d_col int32 in [0, maxq] (pruned entries -1)
+ *   loss, qorder: nullable d_row x d_col; step t of the quantisation loop (same meaning as in obc_prune_trace)
+ *   flags  : OBC_FLAG_OUTLIERS or 0 */
+obc_status obc_quantize(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                        const float *Hinv, int ldhi, float *scale, float *zero, int bits, int symmetric,
+                        const int32_t *prune_order, const int32_t *prune_counts, int flags,
+                        float *W_out, int ldwo, int32_t *codes, float *loss, int32_t *qorder,
+                        int32_t *row_status, void *ws, size_t ws_bytes, obc_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OBC_H_ */

@@ -1,0 +1,206 @@
+"""ctypes binding of libobc.so: one Python function per C entry point, same names, argument marshalling only.
+
+torch is used for device memory (tensors, workspaces) and for the current CUDA stream; every step of the
+method runs inside the library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIBPATH = os.path.join(_HERE, "libobc.so")
+
+OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE = range(6)
+PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
+FLAG_OUTLIERS = 1
+
+EXPORTED_SYMBOLS = (
+    "obc_status_string", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
+    "obc_select_global_mask", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
+)
+
+
+class OBCError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: status {status} ({obc_status_string(status)})")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIBPATH
+
+
+def load_library():
+    """dlopen libobc.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIBPATH):
+        raise RuntimeError(f"{_LIBPATH} is missing: build it with `python -m paper_2208_11580_b200.build` "
+                           "(the CUDA library is the only implementation)")
+    lib = ctypes.CDLL(_LIBPATH)
+    c_int, c_i64, c_sz, c_f, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p
+    lib.obc_status_string.restype = ctypes.c_char_p
+    lib.obc_status_string.argtypes = [c_int]
+    lib.obc_workspace_bytes.restype = c_sz
+    lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
+    lib.obc_hessian.restype = c_int
+    lib.obc_hessian.argtypes = [vp, c_int, c_i64, c_i64, vp, c_int, c_int, c_int, vp, c_sz, vp]
+    lib.obc_hessian_inverse.restype = c_int
+    lib.obc_hessian_inverse.argtypes = [vp, c_int, c_int, c_f, vp, c_int, vp, vp, c_sz, vp]
+    lib.obc_prune_trace.restype = c_int
+    lib.obc_prune_trace.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+    lib.obc_select_global_mask.restype = c_int
+    lib.obc_select_global_mask.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp, c_sz, vp]
+    lib.obc_prune_apply.restype = c_int
+    lib.obc_prune_apply.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, vp, vp, vp, c_int, vp, c_int, vp,
+                                    vp, c_sz, vp]
+    lib.obc_minmax_grid.restype = c_int
+    lib.obc_minmax_grid.argtypes = [vp, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, ctypes.POINTER(c_int), vp]
+    lib.obc_quantize.restype = c_int
+    lib.obc_quantize.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, vp, vp, c_int, c_int, vp, vp, c_int,
+                                 vp, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+    _lib = lib
+    return lib
+
+
+def obc_status_string(status: int) -> str:
+    return load_library().obc_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(t, dtype, name, cuda=True):
+    if t is None:
+        return
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if cuda and not t.is_cuda:
+        raise ValueError(f"{name}: must be a CUDA tensor")
+    if t.dim() >= 1 and t.stride(-1) != 1:
+        raise ValueError(f"{name}: innermost dimension must be contiguous")
+
+
+def _ld(t):
+    return int(t.stride(0)) if t.dim() == 2 and t.shape[0] > 1 else int(t.shape[-1])
+
+
+def obc_workspace_bytes(op: int, row_count: int, d_col: int, n: int = 0) -> int:
+    return int(load_library().obc_workspace_bytes(int(op), int(row_count), int(d_col), int(n)))
+
+
+def _workspace(ws, op, row_count, d_col, n, device, where):
+    need = obc_workspace_bytes(op, row_count, d_col, n)
+    if need == 0:
+        raise OBCError(8, where + " (workspace query)")
+    if ws is None:
+        ws = torch.empty(need, dtype=torch.uint8, device=device)
+    return ws, ws.numel()
+
+
+def _raise(status, where):
+    if status != 0:
+        raise OBCError(status, where)
+
+
+def obc_hessian(X, H, accumulate=False, prec=PREC_FP32, ws=None, stream=None):
+    """H (+)= 2 X X^T for one chunk X (d_col x n) of the calibration data."""
+    _check(X, torch.float32, "X"); _check(H, torch.float32, "H")
+    d, n = X.shape
+    ws, nb = _workspace(ws, OP_HESSIAN, 0, d, n, X.device, "obc_hessian")
+    _raise(load_library().obc_hessian(_ptr(X), d, n, _ld(X), _ptr(H), _ld(H), int(bool(accumulate)), int(prec),
+                                      _ptr(ws), nb, _stream(stream)), "obc_hessian")
+    return H
+
+
+def obc_hessian_inverse(H, damp_rel, Hinv=None, info=None, ws=None, stream=None):
+    """Hinv = inv(H + damp_rel*mean(diag H)*I); returns (Hinv, info) with info a device int32[1]."""
+    _check(H, torch.float32, "H")
+    d = H.shape[0]
+    Hinv = torch.empty_like(H) if Hinv is None else Hinv
+    info = torch.zeros(1, dtype=torch.int32, device=H.device) if info is None else info
+    _check(Hinv, torch.float32, "Hinv"); _check(info, torch.int32, "info")
+    ws, nb = _workspace(ws, OP_INVERSE, 0, d, 0, H.device, "obc_hessian_inverse")
+    _raise(load_library().obc_hessian_inverse(_ptr(H), d, _ld(H), float(damp_rel), _ptr(Hinv), _ld(Hinv), _ptr(info),
+                                              _ptr(ws), nb, _stream(stream)), "obc_hessian_inverse")
+    return Hinv, info
+
+
+def obc_prune_trace(W, Hinv, order, loss, row_status, steps=None, w_trace=None, row_begin=0, row_count=None,
+                    ws=None, stream=None):
+    """Algorithm 1 on rows [row_begin, row_begin+row_count): fills order, loss (and w_trace)."""
+    _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(order, torch.int32, "order")
+    _check(loss, torch.float32, "loss"); _check(row_status, torch.int32, "row_status"); _check(w_trace, torch.float32, "w_trace")
+    R, d = W.shape
+    row_count = R - row_begin if row_count is None else row_count
+    steps = d if steps is None else steps
+    ws, nb = _workspace(ws, OP_PRUNE_TRACE, row_count, d, 0, W.device, "obc_prune_trace")
+    _raise(load_library().obc_prune_trace(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), steps,
+                                          _ptr(order), _ptr(loss), _ptr(w_trace), _ptr(row_status), _ptr(ws), nb,
+                                          _stream(stream)), "obc_prune_trace")
+
+
+def obc_select_global_mask(loss, order, k, counts, mask, ws=None, stream=None):
+    """Algorithm 2: per-row counts and the mask (1 = kept) with k pruned weights."""
+    _check(loss, torch.float32, "loss"); _check(order, torch.int32, "order"); _check(counts, torch.int32, "counts")
+    _check(mask, torch.uint8, "mask")
+    R, d = loss.shape
+    ws, nb = _workspace(ws, OP_SELECT, R, d, 0, loss.device, "obc_select_global_mask")
+    _raise(load_library().obc_select_global_mask(_ptr(loss), _ptr(order), R, d, int(k), _ptr(counts), _ptr(mask),
+                                                 _ptr(ws), nb, _stream(stream)), "obc_select_global_mask")
+
+
+def obc_prune_apply(W, Hinv, order, counts, W_out, row_status, w_trace=None, trace_steps=0, row_begin=0,
+                    row_count=None, ws=None, stream=None):
+    """Weights after the first counts[r] eliminations (trace gather if w_trace is given, else replay)."""
+    _check(W, torch.float32, "W"); _check(W_out, torch.float32, "W_out"); _check(counts, torch.int32, "counts")
+    R, d = W.shape
+    row_count = R - row_begin if row_count is None else row_count
+    if w_trace is None:
+        ws, nb = _workspace(ws, OP_PRUNE_APPLY, row_count, d, 0, W.device, "obc_prune_apply")
+    else:
+        nb = 0 if ws is None else ws.numel()
+    _raise(load_library().obc_prune_apply(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv),
+                                          0 if Hinv is None else _ld(Hinv), _ptr(order), _ptr(counts), _ptr(w_trace),
+                                          int(trace_steps), _ptr(W_out), _ld(W_out), _ptr(row_status), _ptr(ws), nb,
+                                          _stream(stream)), "obc_prune_apply")
+
+
+def obc_minmax_grid(W, bits, symmetric, scale, zero, mask=None, stream=None) -> int:
+    """Per-row min-max grid over kept entries; returns maxq."""
+    _check(W, torch.float32, "W"); _check(scale, torch.float32, "scale"); _check(zero, torch.float32, "zero")
+    _check(mask, torch.uint8, "mask")
+    R, d = W.shape
+    maxq = ctypes.c_int(0)
+    _raise(load_library().obc_minmax_grid(_ptr(W), _ld(W), R, d, _ptr(mask), int(bits), int(bool(symmetric)),
+                                          _ptr(scale), _ptr(zero), ctypes.byref(maxq), _stream(stream)), "obc_minmax_grid")
+    return int(maxq.value)
+
+
+def obc_quantize(W, Hinv, scale, zero, bits, symmetric, W_out, codes, row_status, prune_order=None,
+                 prune_counts=None, flags=0, loss=None, qorder=None, row_begin=0, row_count=None, ws=None, stream=None):
+    """Algorithm 3 (OBQ); with prune_order/prune_counts: replay the pruning first, then quantise survivors."""
+    _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(scale, torch.float32, "scale")
+    _check(zero, torch.float32, "zero"); _check(W_out, torch.float32, "W_out"); _check(codes, torch.int32, "codes")
+    _check(row_status, torch.int32, "row_status"); _check(prune_order, torch.int32, "prune_order")
+    _check(prune_counts, torch.int32, "prune_counts"); _check(loss, torch.float32, "loss"); _check(qorder, torch.int32, "qorder")
+    R, d = W.shape
+    row_count = R - row_begin if row_count is None else row_count
+    ws, nb = _workspace(ws, OP_QUANTIZE, row_count, d, 0, W.device, "obc_quantize")
+    _raise(load_library().obc_quantize(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), _ptr(scale),
+                                       _ptr(zero), int(bits), int(bool(symmetric)), _ptr(prune_order), _ptr(prune_counts),
+                                       int(flags), _ptr(W_out), _ld(W_out), _ptr(codes), _ptr(loss), _ptr(qorder),
+                                       _ptr(row_status), _ptr(ws), nb, _stream(stream)), "obc_quantize")

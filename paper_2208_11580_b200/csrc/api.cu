@@ -1,0 +1,155 @@
+// C ABI of the OBC library: argument checks on the host (nothing is launched or written when they fail),
+// then dispatch to the kernels.  See include/obc.h for the contract of every entry point.
+#include "common.cuh"
+#include <mutex>
+
+namespace obc {
+
+obc_status device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    static bool have[64] = {};
+    int dev = 0;
+    OBC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return OBC_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!have[dev]) {
+        DeviceInfo di;
+        OBC_CUDA_TRY(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        OBC_CUDA_TRY(cudaDeviceGetAttribute(&di.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        OBC_CUDA_TRY(cudaDeviceGetAttribute(&di.l2_bytes, cudaDevAttrL2CacheSize, dev));
+        cache[dev] = di;
+        have[dev] = true;
+    }
+    *out = cache[dev];
+    return OBC_OK;
+}
+
+static bool mat_ok(const void* p, int64_t ld, int64_t min_ld) { return p && ld >= min_ld; }
+static bool mat_aligned(const void* p, int64_t ld) { return aligned16(p) && (ld % 4 == 0); }
+static bool rows_ok(int d_row, int d_col, int row_begin, int row_count) {
+    return d_row > 0 && d_col > 0 && row_begin >= 0 && row_count > 0 && (int64_t)row_begin + row_count <= d_row;
+}
+
+}  // namespace obc
+
+using namespace obc;
+
+extern "C" {
+
+const char* obc_status_string(obc_status s) {
+    switch (s) {
+        case OBC_OK: return "ok";
+        case OBC_ERR_INVALID_ARG: return "invalid argument";
+        case OBC_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+        case OBC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case OBC_ERR_NOT_POSDEF: return "Hessian not positive definite";
+        case OBC_ERR_NONFINITE: return "non-positive or non-finite inverse-Hessian diagonal";
+        case OBC_ERR_TIMEOUT: return "device-side wait timed out";
+        case OBC_ERR_CUDA: return "CUDA runtime error";
+        case OBC_ERR_UNSUPPORTED: return "size not supported";
+    }
+    return "unknown status";
+}
+
+size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
+    if (d_col <= 0 || row_count < 0) return 0;
+    switch (op) {
+        case OBC_OP_HESSIAN: return n > 0 ? hessian_workspace_bytes(d_col, n) : 0;
+        case OBC_OP_INVERSE: return inverse_workspace_bytes(d_col);
+        case OBC_OP_SELECT: return row_count > 0 ? select_workspace_bytes(row_count, d_col) : 0;
+        case OBC_OP_PRUNE_TRACE:
+        case OBC_OP_PRUNE_APPLY:
+        case OBC_OP_QUANTIZE: {
+            DeviceInfo di;
+            if (device_info(&di) != OBC_OK || d_col > OBC_MAX_DCOL) return 0;
+            return engine_workspace_bytes(row_count, d_col, di);
+        }
+    }
+    return 0;
+}
+
+obc_status obc_hessian(const float* X, int d_col, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
+                       obc_prec prec, void* ws, size_t ws_bytes, obc_stream stream) {
+    if (d_col <= 0 || n <= 0 || !mat_ok(X, ldx, n) || !mat_ok(H, ldh, d_col)) return OBC_ERR_INVALID_ARG;
+    if (accumulate != 0 && accumulate != 1) return OBC_ERR_INVALID_ARG;
+    if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
+    if (!mat_aligned(X, ldx) || !mat_aligned(H, ldh)) return OBC_ERR_ALIGNMENT;
+    if (!ws || !aligned256(ws) || ws_bytes < hessian_workspace_bytes(d_col, n)) return OBC_ERR_WORKSPACE;
+    return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, ws, (cudaStream_t)stream);
+}
+
+obc_status obc_hessian_inverse(const float* H, int d_col, int ldh, float damp_rel, float* Hinv, int ldhi,
+                               int32_t* info, void* ws, size_t ws_bytes, obc_stream stream) {
+    if (d_col <= 0 || !mat_ok(H, ldh, d_col) || !mat_ok(Hinv, ldhi, d_col) || !info) return OBC_ERR_INVALID_ARG;
+    if (!(damp_rel >= 0.f)) return OBC_ERR_INVALID_ARG;
+    if (!mat_aligned(H, ldh) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    if (!ws || !aligned256(ws) || ws_bytes < inverse_workspace_bytes(d_col)) return OBC_ERR_WORKSPACE;
+    return inverse_launch(H, d_col, ldh, damp_rel, Hinv, ldhi, info, ws, (cudaStream_t)stream);
+}
+
+obc_status obc_prune_trace(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                           const float* Hinv, int ldhi, int steps, int32_t* order, float* loss, float* w_trace,
+                           int32_t* row_status, void* ws, size_t ws_bytes, obc_stream stream) {
+    if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (steps < 1 || steps > d_col || !order || !loss || !row_status) return OBC_ERR_INVALID_ARG;
+    if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    return engine_prune_trace(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, steps, order, loss, w_trace,
+                              row_status, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+obc_status obc_select_global_mask(const float* loss, const int32_t* order, int d_row, int d_col, int64_t k,
+                                  int32_t* counts, uint8_t* mask, void* ws, size_t ws_bytes, obc_stream stream) {
+    if (d_row <= 0 || d_col <= 0 || !loss || !order || !counts || !mask) return OBC_ERR_INVALID_ARG;
+    if (k < 0 || k > (int64_t)d_row * d_col) return OBC_ERR_INVALID_ARG;
+    if (!ws || !aligned256(ws) || ws_bytes < select_workspace_bytes(d_row, d_col)) return OBC_ERR_WORKSPACE;
+    return select_launch(loss, order, d_row, d_col, k, counts, mask, ws, (cudaStream_t)stream);
+}
+
+obc_status obc_prune_apply(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                           const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts,
+                           const float* w_trace, int trace_steps, float* W_out, int ldwo, int32_t* row_status,
+                           void* ws, size_t ws_bytes, obc_stream stream) {
+    if (!rows_ok(d_row, d_col, row_begin, row_count) || !counts || !mat_ok(W_out, ldwo, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (w_trace) {
+        if (trace_steps < 1 || trace_steps > d_col) return OBC_ERR_INVALID_ARG;
+        return trace_gather_launch(w_trace, trace_steps, counts, d_col, row_begin, row_count, W_out, ldwo,
+                                   (cudaStream_t)stream);
+    }
+    if (!mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col) || !order || !row_status) return OBC_ERR_INVALID_ARG;
+    if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    return engine_replay(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, order, counts, W_out, ldwo,
+                         row_status, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+obc_status obc_minmax_grid(const float* W, int ldw, int d_row, int d_col, const uint8_t* mask, int bits,
+                           int symmetric, float* scale, float* zero, int* maxq_host, obc_stream stream) {
+    if (d_row <= 0 || d_col <= 0 || !mat_ok(W, ldw, d_col) || !scale || !zero) return OBC_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 16 || (symmetric != 0 && symmetric != 1)) return OBC_ERR_INVALID_ARG;
+    if (maxq_host) *maxq_host = grid_maxq(bits, symmetric);
+    return minmax_grid_launch(W, ldw, d_row, d_col, mask, bits, symmetric, scale, zero, (cudaStream_t)stream);
+}
+
+obc_status obc_quantize(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                        const float* Hinv, int ldhi, float* scale, float* zero, int bits, int symmetric,
+                        const int32_t* prune_order, const int32_t* prune_counts, int flags, float* W_out, int ldwo,
+                        int32_t* codes, float* loss, int32_t* qorder, int32_t* row_status, void* ws,
+                        size_t ws_bytes, obc_stream stream) {
+    if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (!scale || !zero || !mat_ok(W_out, ldwo, d_col) || !codes || !row_status) return OBC_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 16 || (symmetric != 0 && symmetric != 1)) return OBC_ERR_INVALID_ARG;
+    if ((prune_order == nullptr) != (prune_counts == nullptr)) return OBC_ERR_INVALID_ARG;
+    if (flags & ~OBC_FLAG_OUTLIERS) return OBC_ERR_INVALID_ARG;
+    if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    return engine_quantize(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, scale, zero, bits, symmetric,
+                           prune_order, prune_counts, flags, W_out, ldwo, codes, loss, qorder, row_status, ws,
+                           ws_bytes, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+"""Shared machinery of the GPU-vs-oracle parity tests (margin-gated, teacher-forced comparison).
+
+The greedy order is chaotic: one flipped pick changes everything after it in that row.  So the oracle is
+run along the order the GPU chose (teacher forcing) and reports, for every step, its own best pick at that
+state and the relative score gap between the forced pick and its best.  A GPU pick passes if it IS the
+oracle's pick, or if that gap is within MARGIN_TOL (a tie within the selection margin).  Loss traces and
+weights are then compared along the common trajectory.
+"""
+import numpy as np
+
+import oracle
+
+MARGIN_TOL = 1e-6      # picks must agree wherever best and forced scores differ by more than this (relative)
+REL_TOL = 1e-4         # loss traces and weights: relative error bound in FP32
+ROUND_TOL = 1e-4       # integer codes may differ only if x/Delta is this close to a rounding boundary
+
+
+def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", scale=None, zero=None, maxq=0,
+               flags=0, gpu_codes=None, gpu_trace=None, steps=None, active0=None):
+    """Compare GPU results for a set of rows with the oracle fed the same FP32 Hinv / W.
+    Returns a dict of statistics; raises AssertionError on a parity violation."""
+    Hinv = np.asarray(Hinv32, dtype=np.float64)
+    W = np.asarray(W32, dtype=np.float64)
+    rows, d = W.shape
+    steps = d if steps is None else steps
+    gpu_order = np.asarray(gpu_order)[:, :steps]
+    res = oracle.run_rows(Hinv, W, steps=steps, mode=mode, scale=scale, zero=zero, maxq=maxq, flags=flags,
+                          forced=gpu_order, active0=active0, want_trace=gpu_trace is not None)
+    assert np.all(res["status"] == 0), f"oracle rejected the GPU order: {res['status']}"
+    differ = res["best"] != gpu_order
+    gap = res["forced_gap"]
+    bad = differ & (gap > MARGIN_TOL)
+    stats = dict(steps=int(rows * steps), picks_differ=int(differ.sum()), max_gap_at_differ=float(gap[differ].max()) if differ.any() else 0.0,
+                 sub_1e5_margin=int((res["margin"] < 1e-5).sum()))
+    assert not bad.any(), (f"{int(bad.sum())} picks differ beyond the margin; first at row/step "
+                           f"{np.argwhere(bad)[0].tolist()}, gap {gap[bad][0]:.3e}")
+    L = res["loss"]
+    gl = np.asarray(gpu_loss, dtype=np.float64)[:, :steps]
+    floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
+    err = np.abs(gl - L) / (np.abs(L) + floor + 1e-300)
+    stats["loss_max_rel"] = float(err.max())
+    assert err.max() <= REL_TOL, f"loss trace off by {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+    if gpu_w is not None:
+        gw = np.asarray(gpu_w, dtype=np.float64)
+        wscale = np.abs(W).max(axis=1, keepdims=True)
+        if mode == "quant" and gpu_codes is not None:
+            gc = np.asarray(gpu_codes)
+            cd = gc != res["codes"]
+            if active0 is not None:
+                cd &= np.asarray(active0, bool)
+            # a differing code is only tolerated where the quotient sat on a rounding boundary
+            rd_by_col = np.full((rows, d), 1.0)
+            np.put_along_axis(rd_by_col, gpu_order.astype(np.int64), res["round_dist"], axis=1)
+            stats["codes_differ"] = int(cd.sum())
+            assert not (cd & (rd_by_col > ROUND_TOL)).any(), "integer codes differ away from rounding boundaries"
+            same = ~cd
+            werr = np.abs(gw - res["w"]) / wscale
+            stats["w_max_rel"] = float(werr[same].max()) if same.any() else 0.0
+            assert werr[same].max() <= REL_TOL
+        else:
+            werr = np.abs(gw - res["w"]) / wscale
+            stats["w_max_rel"] = float(werr.max())
+            assert werr.max() <= REL_TOL, f"weights off by {werr.max():.3e}"
+    if gpu_trace is not None:
+        gt = np.asarray(gpu_trace, dtype=np.float64)
+        wscale = np.abs(W).max(axis=1)[:, None, None]
+        terr = np.abs(gt - res["w_trace"]) / wscale
+        stats["trace_max_rel"] = float(terr.max())
+        assert terr.max() <= REL_TOL
+    stats["oracle"] = res
+    return stats
