@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the ExactOBS / OBQ layer solver on synthetic layers shaped like the paper's workloads.
+
+One "step" is one pass of the whole hot path over one layer, through the C ABI:
+  Hessian (2 X X^T) -> dampened inverse -> per-row elimination (prune trace or OBQ) -> global mask ->
+  final weights (per configuration; see WORKLOADS).
+Prints ONE JSON line.  `value` = eliminated (pruned or quantised) weights per second over the whole job with
+inputs resident in HBM; `e2e` = the same with host<->device copies inside the timed region;
+`roofline` = achieved algorithmic GB/s of the elimination kernel against the measured HBM copy rate;
+`cpu_baseline` = the FP64 oracle on a bounded sample of the same rows on this machine's host cores.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1..C5] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import obc_synth  # noqa: E402
+
+METRIC = "eliminated_weights_per_s"
+UNIT = "weights/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
+    """Algorithmic bytes of `steps` eliminations starting at active size `first`: read + write of the active
+    m x m FP32 block per step = 8 m^2 (the symmetric half actually moved is stated separately)."""
+    first = d if first is None else first
+    steps = first if steps is None else steps
+    m = np.arange(first, first - steps, -1, dtype=np.float64)
+    return int((8.0 * m * m).sum())
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return float(j["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs (read-only)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for nme, v in zip(names, r[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nme)
+            except Exception:
+                pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------------------------
+class Layer:
+    """Device buffers and the stage sequence of one workload, all through the C ABI."""
+
+    def __init__(self, name: str, W: np.ndarray, X: np.ndarray, dev, prec: int):
+        import torch
+        import paper_2208_11580_b200 as obc
+        self.obc, self.torch, self.name, self.dev, self.prec = obc, torch, name, dev, prec
+        self.spec = obc_synth.SPECS[name]
+        self.R, self.d = W.shape
+        self.n = X.shape[1]
+        R, d = self.R, self.d
+        t = torch
+        self.W = t.empty(R, d, dtype=t.float32, device=dev)
+        self.X = t.empty(d, self.n, dtype=t.float32, device=dev)
+        self.H = t.empty(d, d, dtype=t.float32, device=dev)
+        self.Hinv = t.empty(d, d, dtype=t.float32, device=dev)
+        self.info = t.zeros(1, dtype=t.int32, device=dev)
+        self.status = t.zeros(R, dtype=t.int32, device=dev)
+        self.order = t.zeros(R, d, dtype=t.int32, device=dev)
+        self.loss = t.zeros(R, d, dtype=t.float32, device=dev)
+        task = self.spec.task
+        self.trace = None
+        if task in ("prune", "prune+quant"):
+            self.trace = t.empty(R, d + 1, d, dtype=t.float32, device=dev)
+        if task != "quant":
+            self.ks = [obc_synth.pruned_count(R, d, s) for s in self.spec.sparsities]
+            self.counts = [t.zeros(R, dtype=t.int32, device=dev) for _ in self.ks]
+            self.masks = [t.zeros(R, d, dtype=t.uint8, device=dev) for _ in self.ks]
+            self.What = [t.zeros(R, d, dtype=t.float32, device=dev) for _ in self.ks]
+        if task in ("quant", "prune+quant", "compound"):
+            self.scale = t.zeros(R, dtype=t.float32, device=dev)
+            self.zero = t.zeros(R, dtype=t.float32, device=dev)
+            self.Wq = t.zeros(R, d, dtype=t.float32, device=dev)
+            self.codes = t.zeros(R, d, dtype=t.int32, device=dev)
+        need = max(obc.obc_workspace_bytes(obc.OP_HESSIAN, 0, d, self.n), obc.obc_workspace_bytes(obc.OP_INVERSE, 0, d),
+                   obc.obc_workspace_bytes(obc.OP_PRUNE_TRACE, R, d), obc.obc_workspace_bytes(obc.OP_SELECT, R, d))
+        self.ws = t.empty(need, dtype=t.uint8, device=dev)
+        self.W.copy_(t.from_numpy(W))
+        self.X.copy_(t.from_numpy(X))
+        self.engine_ms = []          # (label, CUDA-event ms, algorithmic bytes) per engine launch since reset_timers()
+        self._pending = []
+        self.eliminated = R * d * (2 if task == "prune+quant" else 1)
+
+    def _timed(self, label, nbytes, fn):
+        t = self.torch
+        e0, e1 = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        self._pending.append((label, nbytes, e0, e1))
+
+    def step(self):
+        """Enqueue one pass of the hot path on the current stream (no synchronisation)."""
+        o, R, d, task = self.obc, self.R, self.d, self.spec.task
+        self._timed("hessian", 0, lambda: o.obc_hessian(self.X, self.H, prec=self.prec, ws=self.ws))
+        self._timed("inverse", 0, lambda: o.obc_hessian_inverse(self.H, obc_synth.DAMP_REL, Hinv=self.Hinv, info=self.info, ws=self.ws))
+        full = R * model_bytes_full(d)
+        if task in ("prune", "prune+quant", "compound"):
+            self._timed("engine:prune_trace", full, lambda: o.obc_prune_trace(self.W, self.Hinv, self.order, self.loss, self.status,
+                                                                              w_trace=self.trace, ws=self.ws))
+            for i, k in enumerate(self.ks):
+                self._timed("select", 0, lambda i=i, k=k: o.obc_select_global_mask(self.loss, self.order, k, self.counts[i], self.masks[i], ws=self.ws))
+                if task != "compound":
+                    self._timed("apply", 0, lambda i=i: o.obc_prune_apply(self.W, self.Hinv, self.order, self.counts[i], self.What[i], self.status,
+                                                                           w_trace=self.trace, trace_steps=d, ws=self.ws))
+        if task in ("quant", "prune+quant"):
+            self._timed("grid", 0, lambda: o.obc_minmax_grid(self.W, self.spec.bits, self.spec.symmetric, self.scale, self.zero))
+            self._timed("engine:quantize", full, lambda: o.obc_quantize(self.W, self.Hinv, self.scale, self.zero, self.spec.bits, self.spec.symmetric,
+                                                                        self.Wq, self.codes, self.status, ws=self.ws))
+        if task == "compound":
+            # replay of counts[r] pruning steps + quantisation of the survivors: again every size d..1 once per row
+            self._timed("engine:replay_quantize", full, lambda: o.obc_quantize(
+                self.W, self.Hinv, self.scale, self.zero, self.spec.bits, self.spec.symmetric, self.Wq, self.codes, self.status,
+                prune_order=self.order, prune_counts=self.counts[0], ws=self.ws))
+
+    def reset_timers(self):
+        self._pending = []
+
+    def collect(self):
+        """After a synchronize: CUDA-event milliseconds per stage, summed over the steps since reset_timers()."""
+        out = {}
+        self.engine_ms = []
+        for label, nbytes, e0, e1 in self._pending:
+            ms = e0.elapsed_time(e1)
+            out[label] = out.get(label, 0.0) + ms
+            if label.startswith("engine"):
+                self.engine_ms.append((label, ms, nbytes))
+        return out
+
+    def results_to_host(self, host):
+        """Device->host read of the step's results (final weights / codes / masks) into pinned buffers."""
+        task = self.spec.task
+        n = 0
+        if task != "quant" and task != "compound":
+            for i in range(len(self.ks)):
+                host["What"][i].copy_(self.What[i], non_blocking=True)
+                host["mask"][i].copy_(self.masks[i], non_blocking=True)
+                n += self.What[i].numel() * 4 + self.masks[i].numel()
+        if task in ("quant", "prune+quant", "compound"):
+            host["Wq"].copy_(self.Wq, non_blocking=True)
+            host["codes"].copy_(self.codes, non_blocking=True)
+            n += self.Wq.numel() * 4 + self.codes.numel() * 4
+        return n
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2208_11580_b200 as obc
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    obc.load_library()
+    name = args.workload
+    W, X, spec = obc_synth.make_layer(name)          # every rank compresses its own copy of the layer
+    prec = {"fp32": obc.PREC_FP32, "tf32": obc.PREC_TF32, "bf16x3": obc.PREC_BF16X3}[args.hessian_prec]
+    layer = Layer(name, W, X, dev, prec)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        layer.step()
+    barrier()
+    assert int(layer.info.item()) == 0 and int(layer.status.abs().sum()) == 0, "solver reported a failure status"
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = obc.obc_kernel_launches()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stage_sum, engine_runs = {}, []
+    barrier()
+    layer.reset_timers()
+    ev0.record()
+    for _ in range(args.steps):
+        layer.step()
+    ev1.record()
+    barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    launches = obc.obc_kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    stage_sum = {k: v / args.steps for k, v in layer.collect().items()}     # per-step averages over the timed region
+    engine_runs = list(layer.engine_ms)                                      # every engine launch of the timed region
+    if world > 1:
+        tmax = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms_per_step = total_ms / args.steps
+    value = world * layer.eliminated / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host inputs -> device, hot path, results -> pinned host, every step ---------------------
+    t = torch
+    hW, hX = t.from_numpy(W).pin_memory(), t.from_numpy(X).pin_memory()
+    host = {"What": [], "mask": []}
+    if spec.task not in ("quant", "compound"):
+        host["What"] = [t.empty(layer.R, layer.d, dtype=t.float32).pin_memory() for _ in layer.ks]
+        host["mask"] = [t.empty(layer.R, layer.d, dtype=t.uint8).pin_memory() for _ in layer.ks]
+    if spec.task in ("quant", "prune+quant", "compound"):
+        host["Wq"] = t.empty(layer.R, layer.d, dtype=t.float32).pin_memory()
+        host["codes"] = t.empty(layer.R, layer.d, dtype=t.int32).pin_memory()
+    e2e_steps = max(1, min(args.steps, 2))
+    barrier()
+    layer.reset_timers()
+    ev0.record()
+    d2h = 0
+    for _ in range(e2e_steps):
+        layer.W.copy_(hW, non_blocking=True)
+        layer.X.copy_(hX, non_blocking=True)
+        layer.step()
+        d2h = layer.results_to_host(host)
+    ev1.record()
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        tmax = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    e2e_value = world * layer.eliminated / (e2e_ms / e2e_steps * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = peaks()
+    eng_ms = sum(ms for _, ms, _ in engine_runs)
+    eng_bytes = sum(b for _, _, b in engine_runs)
+    n_eng = max(1, len(engine_runs))
+    achieved = eng_bytes / (eng_ms * 1e-3) / 1e9 if eng_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "row_engine_kernel", "achieved": round(achieved, 1), "peak": peak,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": None,
+                "algorithmic_bytes_per_launch": eng_bytes // n_eng, "ms_per_launch": round(eng_ms / n_eng, 3),
+                "launches_timed": len(engine_runs),
+                "note": "algorithmic bytes = 8 m^2 per elimination step (full active block read+write); the kernel "
+                        "moves only the lower triangle (4 m^2), so frac can exceed 1 without re-use"}
+    cpu = cpu_baseline(name, W, layer.Hinv.cpu().numpy(), layer, args.cpu_seconds)
+    out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": f"{name}: {spec.note}", "d_row": layer.R, "d_col": layer.d, "n_calib": layer.n,
+                      "task": spec.task, "bits": spec.bits, "sparsities": list(spec.sparsities),
+                      "hessian_prec": args.hessian_prec, "damp_rel": obc_synth.DAMP_REL,
+                      "l2": "per-row inverse-Hessian working set exceeds L2 (inputs larger than L2)"
+                            if layer.R * layer.d * layer.d * 2 > 126e6 else "working set fits L2 (small case)",
+                      "parallelism": f"rows of one layer per GPU; {world} independent layer(s)"},
+           "stage_ms": {k: round(v, 3) for k, v in stage_sum.items()},
+           "clocks": clocks, "gpu_launches": int(launches),
+           "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(hW.numel() * 4 + hX.numel() * 4),
+                   "d2h_bytes_per_step": int(d2h), "ms_per_step": round(e2e_ms / e2e_steps, 3), "steps": e2e_steps},
+           "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(name, W, Hinv32, layer, budget_s):
+    """FP64 oracle on a bounded row sample of the same workload (rows only), on this machine's host cores."""
+    import oracle
+    spec = obc_synth.SPECS[name]
+    cores = oracle.threads()
+    d = W.shape[1]
+    # ~1.5e-9 s per inner update on one core (measured order of magnitude); rows sized to the budget
+    est_row = 1.5e-9 * (2.0 / 3.0) * d ** 3 + 1e-4
+    rows = int(max(1, min(W.shape[0], cores * max(1, int(budget_s / est_row)))))
+    Hinv = Hinv32.astype(np.float64)
+    Ws = W[:rows]
+    kw = {}
+    if spec.task == "quant":
+        sc, ze, mq = oracle.minmax_grid(Ws, spec.bits, spec.symmetric)
+        kw = dict(mode="quant", scale=sc, zero=ze, maxq=mq)
+    t0 = time.perf_counter()
+    oracle.run_rows(Hinv, Ws, **kw)
+    dt = time.perf_counter() - t0
+    return {"value": round(rows * d / dt, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{rows} of {W.shape[0]} rows of {name}, elimination loop only (Hessian/inverse excluded), "
+                      f"{dt:.1f} s, OpenMP over rows", "seconds": round(dt, 2)}
+
+
+def run_reference(args):
+    """The FP64 oracle as it stands, timed on host cores: each step = the elimination loop on a bounded sample of rows."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    name = args.workload
+    W, X, spec = obc_synth.make_layer(name)
+    d = W.shape[1]
+    H = oracle.hessian(X)
+    Hinv, info = oracle.inverse(H, obc_synth.DAMP_REL)
+    assert info == 0
+    cores = oracle.threads()
+    est_row = 1.5e-9 * (2.0 / 3.0) * d ** 3 + 1e-4
+    per_step_budget = max(2.0, 60.0 / max(1, args.steps + args.warmup))
+    rows = int(max(1, min(W.shape[0], cores * max(1, int(per_step_budget / est_row)))))
+    kw = {}
+    if spec.task == "quant":
+        sc, ze, mq = oracle.minmax_grid(W[:rows], spec.bits, spec.symmetric)
+        kw = dict(mode="quant", scale=sc, zero=ze, maxq=mq)
+    for _ in range(args.warmup):
+        oracle.run_rows(Hinv, W[:rows], **kw)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.run_rows(Hinv, W[:rows], **kw)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = rows * d / dt
+    sample = f"{rows} of {W.shape[0]} rows of {name} per step, elimination loop only, OpenMP over rows"
+    out = {"impl": "reference", "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{name}: {spec.note}", "d_row": W.shape[0], "d_col": d, "n_calib": X.shape[1],
+                      "task": spec.task},
+           "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="C3", choices=sorted(obc_synth.SPECS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--hessian-prec", default="fp32", choices=["fp32", "tf32", "bf16x3"])
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -65,6 +65,9 @@ typedef void *obc_stream;      /* a cudaStream_t (NULL = default stream) */
 
 const char *obc_status_string(obc_status s);
 
+/* Diagnostic (host function): number of kernels this library has launched in the calling process so far. */
+unsigned long long obc_kernel_launches(void);
+
 /* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).
  * n is only used by OBC_OP_HESSIAN; row_count (the rows one call processes) by the three row-engine ops,
  * where 0 means "size for any row_count".  Returns 0 on invalid arguments. */

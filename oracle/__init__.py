@@ -83,7 +83,7 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
              forced=None, active0=None, want_trace=False):
     """Algorithm 1 (mode='prune') / Algorithm 3 (mode='quant') on every row of W with the shared Hinv.
 
-    Returns a dict: order, loss, margin, best, forced_gap, round_dist (rows x steps), w (rows x d final
+    Returns a dict: order, loss, margin, best, forced_gap, round_dist, pivot_diag (rows x steps), w (rows x d final
     weights), codes (rows x d, quant only), w_trace (rows x (steps+1) x d if want_trace), status (rows).
     """
     Hinv = np.ascontiguousarray(Hinv, dtype=np.float64)
@@ -104,6 +104,7 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
         order=np.full((rows, steps), -1, np.int32), loss=np.zeros((rows, steps)),
         margin=np.ones((rows, steps)), best=np.full((rows, steps), -1, np.int32),
         forced_gap=np.zeros((rows, steps)), round_dist=np.full((rows, steps), 0.5),
+        pivot_diag=np.zeros((rows, steps)),
         codes=np.full((rows, d), -1, np.int32), status=np.zeros(rows, np.int32),
         w_trace=np.zeros((rows, steps + 1, d)) if want_trace else None)
     I32, F64, U8 = ctypes.c_int32, ctypes.c_double, ctypes.c_uint8
@@ -111,7 +112,7 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
                      ctypes.c_int(m), _p(sc, F64), _p(ze, F64), ctypes.c_int(int(maxq)), ctypes.c_int(int(flags)),
                      _p(fo, I32), _p(a0, U8), _p(out["order"], I32), _p(out["loss"], F64),
                      _p(out["margin"], F64), _p(out["best"], I32), _p(out["forced_gap"], F64),
-                     _p(out["round_dist"], F64), _p(out["w_trace"], F64), _p(out["codes"], I32),
+                     _p(out["round_dist"], F64), _p(out["pivot_diag"], F64), _p(out["w_trace"], F64), _p(out["codes"], I32),
                      _p(out["status"], I32))
     out["w"] = Wd
     return out
@@ -130,7 +131,7 @@ def eliminate_one_row(Hinv, w, **kw):
     a0 = None if a0 is None else np.ascontiguousarray(a0, dtype=np.uint8)
     order = np.full(steps, -1, np.int32); loss = np.zeros(steps); margin = np.ones(steps)
     best = np.full(steps, -1, np.int32); gap = np.zeros(steps); rd = np.full(steps, 0.5)
-    codes = np.full(d, -1, np.int32); trace = np.zeros((steps + 1, d))
+    codes = np.full(d, -1, np.int32); trace = np.zeros((steps + 1, d)); pdg = np.zeros(steps)
     I32, F64, U8 = ctypes.c_int32, ctypes.c_double, ctypes.c_uint8
     lib = _L()
     lib.oracle_row.restype = ctypes.c_int
@@ -138,9 +139,9 @@ def eliminate_one_row(Hinv, w, **kw):
                         ctypes.c_double(float(kw.get("scale", 1.0))), ctypes.c_double(float(kw.get("zero", 0.0))),
                         ctypes.c_int(int(kw.get("maxq", 0))), ctypes.c_int(int(kw.get("flags", 0))),
                         _p(fo, I32), _p(a0, U8), _p(order, I32), _p(loss, F64), _p(margin, F64), _p(best, I32),
-                        _p(gap, F64), _p(rd, F64), _p(trace, F64), _p(codes, I32))
+                        _p(gap, F64), _p(rd, F64), _p(pdg, F64), _p(trace, F64), _p(codes, I32))
     return dict(Hi=Hi, w=wd, order=order, loss=loss, margin=margin, best=best, forced_gap=gap,
-                round_dist=rd, codes=codes, w_trace=trace, status=int(st))
+                round_dist=rd, pivot_diag=pdg, codes=codes, w_trace=trace, status=int(st))
 
 
 def global_mask(loss, order, k: int):

@@ -111,14 +111,15 @@ static double grid_quant(double x, double scale, double zero, int maxq)
  * |q(w_j)-w_j| > Delta/2, the one with the largest such error is taken first (ties: lowest index).
  *
  * active0 (nullable): 1 = in M at the start.  Hi is the row's private d x d copy of Hinv and is
- * modified in place (so the caller can inspect it).  w_trace (nullable) is (steps+1) x d with
+ * modified in place (so the caller can inspect it).  pivot_diag[t] (nullable) records [Hinv]_pp of step t.
+ * w_trace (nullable) is (steps+1) x d with
  * w_trace[0] = w on entry.  Returns 0, or 1+t if [Hinv]_pp was not positive and finite at step t.
  */
 int oracle_row(double *Hi, int d, double *w, int steps, int mode,
                double scale, double zero, int maxq, int flags,
                const int32_t *forced, const uint8_t *active0,
                int32_t *order, double *loss, double *margin, int32_t *best, double *forced_gap,
-               double *round_dist, double *w_trace, int32_t *codes)
+               double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes)
 {
     const double tiny = 1e-300;
     int32_t *M = (int32_t *)malloc((size_t)d * sizeof(int32_t));   /* the remaining set, ascending */
@@ -176,6 +177,7 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
         if (forced_gap) forced_gap[t] = (sp - sb) / fmax(sp, tiny);
         order[t] = p;
         loss[t] = sp;
+        if (pivot_diag) pivot_diag[t] = dpp;
         const double qp = mode ? grid_quant(w[p], scale, zero, maxq) : 0.0;
         if (mode) {
             const double xq = w[p] / scale;
@@ -208,14 +210,14 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
 }
 
 /* Many independent rows (Section 3: no Hessian interaction between rows); OpenMP over rows.
- * Per-row arrays are strided by `steps` (order, loss, margin, best, forced_gap, round_dist),
+ * Per-row arrays are strided by `steps` (order, loss, margin, best, forced_gap, round_dist, pivot_diag),
  * by d (w, codes, active0) and by (steps+1)*d (w_trace).  scale/zero are per row.  Each row works on
  * its own copy of Hinv.  status[r] receives oracle_row's return value. */
 void oracle_rows(const double *Hinv, int d, int rows, double *W, int steps, int mode,
                  const double *scale, const double *zero, int maxq, int flags,
                  const int32_t *forced, const uint8_t *active0,
                  int32_t *order, double *loss, double *margin, int32_t *best, double *forced_gap,
-                 double *round_dist, double *w_trace, int32_t *codes, int32_t *status)
+                 double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes, int32_t *status)
 {
 #pragma omp parallel for schedule(dynamic, 1)
     for (int r = 0; r < rows; ++r) {
@@ -227,6 +229,7 @@ void oracle_rows(const double *Hinv, int d, int rows, double *W, int steps, int 
                                forced ? forced + so : NULL, active0 ? active0 + (int64_t)r * d : NULL,
                                order + so, loss + so, margin ? margin + so : NULL, best ? best + so : NULL,
                                forced_gap ? forced_gap + so : NULL, round_dist ? round_dist + so : NULL,
+                               pivot_diag ? pivot_diag + so : NULL,
                                w_trace ? w_trace + (int64_t)r * (steps + 1) * d : NULL,
                                codes ? codes + (int64_t)r * d : NULL);
         free(Hi);

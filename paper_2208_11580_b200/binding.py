@@ -18,7 +18,7 @@ PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
 FLAG_OUTLIERS = 1
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
+    "obc_status_string", "obc_kernel_launches", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
     "obc_select_global_mask", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -48,6 +48,8 @@ def load_library():
     c_int, c_i64, c_sz, c_f, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_float, ctypes.c_void_p
     lib.obc_status_string.restype = ctypes.c_char_p
     lib.obc_status_string.argtypes = [c_int]
+    lib.obc_kernel_launches.restype = ctypes.c_ulonglong
+    lib.obc_kernel_launches.argtypes = []
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
@@ -72,6 +74,10 @@ def load_library():
 
 def obc_status_string(status: int) -> str:
     return load_library().obc_status_string(int(status)).decode()
+
+
+def obc_kernel_launches() -> int:
+    return int(load_library().obc_kernel_launches())
 
 
 def _ptr(t):
@@ -130,7 +136,8 @@ def obc_hessian_inverse(H, damp_rel, Hinv=None, info=None, ws=None, stream=None)
     """Hinv = inv(H + damp_rel*mean(diag H)*I); returns (Hinv, info) with info a device int32[1]."""
     _check(H, torch.float32, "H")
     d = H.shape[0]
-    Hinv = torch.empty_like(H) if Hinv is None else Hinv
+    if Hinv is None:   # leading dimension padded to a multiple of 4 floats
+        Hinv = torch.empty(d, (d + 3) // 4 * 4, dtype=torch.float32, device=H.device)[:, :d]
     info = torch.zeros(1, dtype=torch.int32, device=H.device) if info is None else info
     _check(Hinv, torch.float32, "Hinv"); _check(info, torch.int32, "info")
     ws, nb = _workspace(ws, OP_INVERSE, 0, d, 0, H.device, "obc_hessian_inverse")

@@ -1,9 +1,13 @@
 // C ABI of the OBC library: argument checks on the host (nothing is launched or written when they fail),
 // then dispatch to the kernels.  See include/obc.h for the contract of every entry point.
 #include "common.cuh"
+#include <atomic>
 #include <mutex>
 
 namespace obc {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 obc_status device_info(DeviceInfo* out) {
     static std::mutex mu;
@@ -51,6 +55,8 @@ const char* obc_status_string(obc_status s) {
     }
     return "unknown status";
 }
+
+unsigned long long obc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
     if (d_col <= 0 || row_count < 0) return 0;

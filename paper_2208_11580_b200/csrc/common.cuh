@@ -13,6 +13,9 @@
 
 namespace obc {
 
+// Every kernel launch of the library goes through this counter (read by obc_kernel_launches()).
+void count_launch(int n = 1);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

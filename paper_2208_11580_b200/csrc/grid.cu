@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(GRID_THREADS) trace_gather_kernel(const float*
 obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const uint8_t* mask, int bits, int symmetric,
                               float* scale, float* zero, cudaStream_t stream) {
     minmax_grid_kernel<<<rows, GRID_THREADS, 0, stream>>>(W, ldw, d, mask, bits, symmetric, scale, zero);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
@@ -52,6 +53,7 @@ obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const ui
 obc_status trace_gather_launch(const float* w_trace, int trace_steps, const int32_t* counts, int d, int row_begin,
                                int row_count, float* W_out, int ldwo, cudaStream_t stream) {
     trace_gather_kernel<<<row_count, GRID_THREADS, 0, stream>>>(w_trace, trace_steps, counts, d, row_begin, W_out, ldwo);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

@@ -116,6 +116,7 @@ obc_status hessian_finalize_launch(const float* partial, int splits, int d, floa
                                    cudaStream_t stream) {
     dim3 grid((d + 255) / 256, d);
     hessian_finalize_kernel<<<grid, 256, 0, stream>>>(partial, splits, d, H, ldh, accumulate);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
@@ -129,6 +130,7 @@ obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, fl
     dim3 grid(T * (T + 1) / 2, splits);
     float* partial = reinterpret_cast<float*>(ws);
     syrk_fp32_kernel<<<grid, 256, 0, stream>>>(X, d, n, ldx, slice, partial);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, stream);
 }

@@ -79,6 +79,7 @@ static void dgemm(cudaStream_t s, int M, int N, int K, double alpha, const doubl
     if (M <= 0 || N <= 0) return;
     dim3 grid((N + GT - 1) / GT, (M + GT - 1) / GT);
     dgemm_kernel<TA, TB><<<grid, 256, 0, s>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, lower_only, k_lo);
+    count_launch();
 }
 
 // trace of H (FP32) -> lambda; single block
@@ -202,14 +203,18 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
     double* lambda = reinterpret_cast<double*>(p);
 
     damp_kernel<<<1, 256, 0, s>>>(H, ldh, d, damp_rel, lambda, info);
+    count_launch();
     widen_kernel<<<592, 256, 0, s>>>(H, ldh, d, lambda, A, Li);
+    count_launch();
     // blocked Cholesky, lower, in place
     for (int k0 = 0; k0 < d; k0 += NB) {
         const int nb = d - k0 < NB ? d - k0 : NB;
         chol_diag_kernel<<<1, 256, 0, s>>>(A, Li, d, k0, nb, info);
+        count_launch();
         const int below = d - k0 - nb;
         if (below > 0) {
             chol_panel_kernel<<<(below + GT - 1) / GT, 256, 0, s>>>(A, Li, d, k0, nb);
+            count_launch();
             const double* P = A + (size_t)(k0 + nb) * d + k0;
             dgemm<false, true>(s, below, below, nb, -1.0, P, d, P, d, 1.0, A + (size_t)(k0 + nb) * d + k0 + nb, d, 1, 0);
         }
@@ -223,6 +228,7 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
     // C = Li^T Li on the lower tiles, then mirror into FP32
     dgemm<true, false>(s, d, d, d, 1.0, Li, d, Li, d, 0.0, C, d, 1, 1);
     narrow_kernel<<<592, 256, 0, s>>>(C, d, Hinv, ldhi);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

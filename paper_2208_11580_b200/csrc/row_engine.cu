@@ -435,6 +435,7 @@ obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t s
     const size_t smem = engine_smem_bytes(a.cap, a.ms);
     OBC_CUDA_TRY(cudaFuncSetAttribute(row_engine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     row_engine_kernel<<<blocks, ENGINE_THREADS, smem, stream>>>(a);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

@@ -167,17 +167,24 @@ obc_status select_launch(const float* loss, const int32_t* order, int rows, int 
     int* eq = reinterpret_cast<int*>(p);
     const long long n = (long long)rows * d;
     prefix_max_kernel<<<rows, SEL_THREADS, 0, stream>>>(loss, d, keys);
+    count_launch();
     select_init_kernel<<<1, 256, 0, stream>>>(st, (long long)k);
+    count_launch();
     int hb = (int)((n + SEL_THREADS * 8 - 1) / (SEL_THREADS * 8));
     if (hb > 1184) hb = 1184;
     if (hb < 1) hb = 1;
     for (int shift = 24; shift >= 0; shift -= 8) {
         select_hist_kernel<<<hb, SEL_THREADS, 0, stream>>>(keys, n, shift, st);
+        count_launch();
         select_pick_kernel<<<1, 256, 0, stream>>>(st, shift);
+        count_launch();
     }
     select_count_kernel<<<rows, SEL_THREADS, 0, stream>>>(keys, d, st, lt, eq);
+    count_launch();
     select_ties_kernel<<<1, SEL_THREADS, 0, stream>>>(st, lt, eq, rows, counts);
+    count_launch();
     mask_kernel<<<rows, SEL_THREADS, 0, stream>>>(order, counts, d, mask);
+    count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }

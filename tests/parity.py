@@ -37,6 +37,11 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
     L = res["loss"]
     gl = np.asarray(gpu_loss, dtype=np.float64)[:, :steps]
     floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
+    if mode == "quant":
+        # the quantisation loss is a squared DIFFERENCE w - q(w): an absolute weight error within the weight
+        # tolerance moves it by up to ~REL_TOL of the loss of a half-step error at that pivot
+        half = 0.5 * np.broadcast_to(np.asarray(scale, dtype=np.float64), (rows,))[:, None]
+        floor = np.maximum(floor, half * half / res["pivot_diag"])
     err = np.abs(gl - L) / (np.abs(L) + floor + 1e-300)
     stats["loss_max_rel"] = float(err.max())
     assert err.max() <= REL_TOL, f"loss trace off by {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
