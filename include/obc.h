@@ -44,7 +44,8 @@ typedef enum {
     OBC_ERR_NONFINITE = 5,     /* (reported through row_status[]) non-positive / non-finite [Hinv]_pp    */
     OBC_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired                                     */
     OBC_ERR_CUDA = 7,          /* a CUDA runtime call failed (launch configuration, missing device ...)  */
-    OBC_ERR_UNSUPPORTED = 8    /* size outside what the kernels support (d_col > OBC_MAX_DCOL)           */
+    OBC_ERR_UNSUPPORTED = 8,   /* size outside what the kernels support (d_col > OBC_MAX_DCOL)           */
+    OBC_ERR_STATIC_SCRATCH = 9 /* problem larger than the built-in scratch area of a *_static entry point */
 } obc_status;
 
 typedef enum { OBC_PREC_FP32 = 0, OBC_PREC_TF32 = 1, OBC_PREC_BF16X3 = 2 } obc_prec;
@@ -111,6 +112,25 @@ obc_status obc_prune_trace(const float *W, int ldw, int d_row, int d_col, int ro
 obc_status obc_select_global_mask(const float *loss, const int32_t *order, int d_row, int d_col, int64_t k,
                                   int32_t *counts, uint8_t *mask,
                                   void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Allocation-free variant of obc_select_global_mask.  The paper has no counterpart: this exists for callers
+ * that cannot provide a workspace because they are not allowed to allocate device memory at this point --
+ * for example a plug-in running inside a host application that handed the whole GPU to its own memory pool at
+ * start-up, or a service loop where a cudaMalloc (which may synchronise the device and can fail under
+ * fragmentation) is not acceptable once it is running.  Inputs and outputs are still the caller's; the scratch
+ * memory is a fixed array inside the library's device image, so every GPU that loads the library carries it
+ * (about 16.2 MiB) until the process exits.
+ *   Limits: d_row <= OBC_SELECT_STATIC_MAX_ROWS and d_row*d_col <= OBC_SELECT_STATIC_MAX_KEYS; anything larger
+ *   returns OBC_ERR_STATIC_SCRATCH and launches nothing.
+ *   The first call on each device looks up the array's device address (a host-side runtime call, no allocation);
+ *   make that first call outside any stream capture.  No call allocates or frees memory.
+ *   All calls on a device share the one array: the call rewrites everything it later reads, so back-to-back calls
+ *   on one stream are fine, but two calls that can overlap on the GPU (different streams or threads) race.
+ * Results are identical to obc_select_global_mask. */
+#define OBC_SELECT_STATIC_MAX_KEYS (4 * 1024 * 1024)
+#define OBC_SELECT_STATIC_MAX_ROWS 16384
+obc_status obc_select_global_mask_static(const float *loss, const int32_t *order, int d_row, int d_col, int64_t k,
+                                         int32_t *counts, uint8_t *mask, obc_stream stream);
 
 /* Section 3 / Figure 1: the weights of each row after its first counts[r] eliminations.
  * w_trace != NULL (layout of obc_prune_trace with this `trace_steps`): rows are gathered from the trace.

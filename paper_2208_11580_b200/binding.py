@@ -19,7 +19,7 @@ FLAG_OUTLIERS = 1
 
 EXPORTED_SYMBOLS = (
     "obc_status_string", "obc_kernel_launches", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
-    "obc_select_global_mask", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
+    "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
 
@@ -60,6 +60,8 @@ def load_library():
     lib.obc_prune_trace.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
     lib.obc_select_global_mask.restype = c_int
     lib.obc_select_global_mask.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp, c_sz, vp]
+    lib.obc_select_global_mask_static.restype = c_int
+    lib.obc_select_global_mask_static.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp]
     lib.obc_prune_apply.restype = c_int
     lib.obc_prune_apply.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, vp, vp, vp, c_int, vp, c_int, vp,
                                     vp, c_sz, vp]
@@ -168,6 +170,17 @@ def obc_select_global_mask(loss, order, k, counts, mask, ws=None, stream=None):
     ws, nb = _workspace(ws, OP_SELECT, R, d, 0, loss.device, "obc_select_global_mask")
     _raise(load_library().obc_select_global_mask(_ptr(loss), _ptr(order), R, d, int(k), _ptr(counts), _ptr(mask),
                                                  _ptr(ws), nb, _stream(stream)), "obc_select_global_mask")
+
+
+def obc_select_global_mask_static(loss, order, k, counts, mask, stream=None):
+    """Algorithm 2 without a workspace: for callers that must not allocate device memory.  Uses the scratch array
+    built into the library (limits: OBC_SELECT_STATIC_MAX_ROWS rows, OBC_SELECT_STATIC_MAX_KEYS entries); calls that
+    may overlap on the GPU must not share a device.  Same results as obc_select_global_mask."""
+    _check(loss, torch.float32, "loss"); _check(order, torch.int32, "order"); _check(counts, torch.int32, "counts")
+    _check(mask, torch.uint8, "mask")
+    R, d = loss.shape
+    _raise(load_library().obc_select_global_mask_static(_ptr(loss), _ptr(order), R, d, int(k), _ptr(counts), _ptr(mask),
+                                                        _stream(stream)), "obc_select_global_mask_static")
 
 
 def obc_prune_apply(W, Hinv, order, counts, W_out, row_status, w_trace=None, trace_steps=0, row_begin=0,

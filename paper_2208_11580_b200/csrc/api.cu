@@ -52,6 +52,7 @@ const char* obc_status_string(obc_status s) {
         case OBC_ERR_TIMEOUT: return "device-side wait timed out";
         case OBC_ERR_CUDA: return "CUDA runtime error";
         case OBC_ERR_UNSUPPORTED: return "size not supported";
+        case OBC_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch area of this allocation-free entry point";
     }
     return "unknown status";
 }

@@ -10,6 +10,7 @@
 // Kernels: prefix-max keys -> 4-pass 8-bit radix select of the k-th key T -> per-row counts -> tie
 // distribution over rows -> mask scatter.  Keys are non-negative floats compared as unsigned integers.
 #include "common.cuh"
+#include <mutex>
 
 namespace obc {
 
@@ -189,4 +190,46 @@ obc_status select_launch(const float* loss, const int32_t* order, int rows, int 
     return OBC_OK;
 }
 
+// ---- allocation-free variant ----------------------------------------------------------------------------------
+// Scratch for obc_select_global_mask_static: a fixed array in device memory that every GPU loading this library
+// holds until the process exits.  Sized for OBC_SELECT_STATIC_MAX_KEYS loss entries and
+// OBC_SELECT_STATIC_MAX_ROWS rows (16 MiB of keys + 128 KiB of per-row counters + the selection state).
+constexpr size_t SELECT_STATIC_BYTES =
+    ((size_t)OBC_SELECT_STATIC_MAX_KEYS * 4 + 255) / 256 * 256 + (sizeof(SelectState) + 255) / 256 * 256 +
+    2 * (((size_t)OBC_SELECT_STATIC_MAX_ROWS * 4 + 255) / 256 * 256);
+static __device__ __align__(256) unsigned char g_select_scratch[SELECT_STATIC_BYTES];
+
+// Device address of the array on the CURRENT device.  In host code the array's name is only a stand-in, so
+// the address is looked up once per device (with that device current) and cached.
+static obc_status select_static_scratch(void** out) {
+    static std::mutex mu;
+    static void* ptrs[64] = {};
+    int dev = 0;
+    OBC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return OBC_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        OBC_CUDA_TRY(cudaGetSymbolAddress(&p, g_select_scratch));
+        if (!p) return OBC_ERR_CUDA;
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return OBC_OK;
+}
+
 }  // namespace obc
+
+extern "C" obc_status obc_select_global_mask_static(const float* loss, const int32_t* order, int d_row, int d_col,
+                                                    int64_t k, int32_t* counts, uint8_t* mask, obc_stream stream) {
+    using namespace obc;
+    if (d_row <= 0 || d_col <= 0 || !loss || !order || !counts || !mask) return OBC_ERR_INVALID_ARG;
+    if (k < 0 || k > (int64_t)d_row * d_col) return OBC_ERR_INVALID_ARG;
+    if (d_row > OBC_SELECT_STATIC_MAX_ROWS || (int64_t)d_row * d_col > (int64_t)OBC_SELECT_STATIC_MAX_KEYS)
+        return OBC_ERR_STATIC_SCRATCH;
+    void* scratch = nullptr;
+    const obc_status st = select_static_scratch(&scratch);
+    if (st != OBC_OK) return st;
+    // every launch sequence re-initialises the selection state and overwrites the keys / counters it reads
+    return select_launch(loss, order, d_row, d_col, k, counts, mask, scratch, (cudaStream_t)stream);
+}

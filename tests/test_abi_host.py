@@ -27,8 +27,8 @@ def test_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     from paper_2208_11580_b200 import obc_status_string
-    seen = {obc_status_string(i) for i in range(9)}
-    assert len(seen) == 9 and "ok" in seen
+    seen = {obc_status_string(i) for i in range(10)}
+    assert len(seen) == 10 and "ok" in seen
     assert obc_status_string(12345) == "unknown status"
 
 
@@ -55,6 +55,10 @@ def test_argument_errors_return_before_any_launch(lib):
     assert lib.obc_select_global_mask(good, good, 4, 8, 33, good, good, good, 1 << 30, None) == 1   # k > d_row*d_col
     assert lib.obc_select_global_mask(good, good, 4, 8, -1, good, good, good, 1 << 30, None) == 1
     assert lib.obc_select_global_mask(good, good, 4, 8, 5, good, good, good, 8, None) == 3
+    st = lib.obc_select_global_mask_static
+    assert st(good, good, 4, 8, 33, good, good, None) == 1                                           # k out of range
+    assert st(good, good, 20000, 8, 5, good, good, None) == 9                                        # rows over the built-in limit
+    assert st(good, good, 4096, 2048, 5, good, good, None) == 9                                      # entries over the limit
     assert lib.obc_minmax_grid(good, 8, 4, 8, None, 1, 0, good, good, None, None) == 1              # bits
     assert lib.obc_minmax_grid(good, 8, 4, 8, None, 4, 2, good, good, None, None) == 1              # symmetric flag
     q = lib.obc_quantize
