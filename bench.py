@@ -31,6 +31,10 @@ import obc_synth  # noqa: E402
 METRIC = "eliminated_weights_per_s"
 UNIT = "weights/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per algorithmic byte of the row engine, from the ncu capture summarised in
+# profiles/row_engine_d1152_rows148_ncu_full.txt (287.8 GB moved for 603.3 GB of 8 m^2 model bytes); the
+# traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
+ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 287.8 / 603.3
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
@@ -295,7 +299,9 @@ def run_ours(args):
     n_eng = max(1, len(engine_runs))
     achieved = eng_bytes / (eng_ms * 1e-3) / 1e9 if eng_ms > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "row_engine_kernel", "achieved": round(achieved, 1), "peak": peak,
-                "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": None,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "traffic": int(eng_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
+                "traffic_source": "scaled from the d=1152 x 148-row ncu capture by algorithmic bytes",
                 "algorithmic_bytes_per_launch": eng_bytes // n_eng, "ms_per_launch": round(eng_ms / n_eng, 3),
                 "launches_timed": len(engine_runs),
                 "note": "algorithmic bytes = 8 m^2 per elimination step (full active block read+write); the kernel "
