@@ -394,7 +394,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C3", choices=sorted(obc_synth.SPECS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--hessian-prec", default="fp32", choices=["fp32", "tf32", "bf16x3"])
+    ap.add_argument("--hessian-prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":

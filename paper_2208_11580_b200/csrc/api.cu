@@ -83,7 +83,8 @@ obc_status obc_hessian(const float* X, int d_col, int64_t n, int64_t ldx, float*
     if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
     if (!mat_aligned(X, ldx) || !mat_aligned(H, ldh)) return OBC_ERR_ALIGNMENT;
     if (!ws || !aligned256(ws) || ws_bytes < hessian_workspace_bytes(d_col, n)) return OBC_ERR_WORKSPACE;
-    return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, ws, (cudaStream_t)stream);
+    if (prec == OBC_PREC_FP32) return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, ws, (cudaStream_t)stream);
+    return hessian_tc_launch(X, d_col, n, ldx, H, ldh, accumulate, prec, ws, (cudaStream_t)stream);
 }
 
 obc_status obc_hessian_inverse(const float* H, int d_col, int ldh, float damp_rel, float* Hinv, int ldhi,

@@ -67,6 +67,8 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
                           void* ws, cudaStream_t s);
 obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
                                void* ws, cudaStream_t stream);
+obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
+                             obc_prec prec, void* ws, cudaStream_t stream);
 obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const uint8_t* mask, int bits, int symmetric,
                               float* scale, float* zero, cudaStream_t stream);
 obc_status trace_gather_launch(const float* w_trace, int trace_steps, const int32_t* counts, int d, int row_begin,

@@ -19,7 +19,7 @@ int hessian_splits(int d, int64_t n) {
     const int T = (d + HT - 1) / HT;
     const int ntiles = T * (T + 1) / 2;
     int64_t s = (444 + ntiles - 1) / ntiles;
-    const int64_t by_len = (n + 8191) / 8192;
+    const int64_t by_len = (n + 2047) / 2048;      // short accumulation chains: partial sums are combined in FP32 RN
     if (by_len > s) s = by_len;
     if (s > 32) s = 32;
     if (s * 64 > n) s = n / 64;
@@ -27,8 +27,10 @@ int hessian_splits(int d, int64_t n) {
     return (int)s;
 }
 
-size_t hessian_workspace_bytes(int d, int64_t n) {
-    return round_up((size_t)hessian_splits(d, n) * d * d * sizeof(float), 256);
+size_t hessian_tc_extra_bytes(int d, int64_t n);
+
+size_t hessian_workspace_bytes(int d, int64_t n) {      // partial sums + what the tensor-core paths add
+    return round_up((size_t)hessian_splits(d, n) * d * d * sizeof(float), 256) + hessian_tc_extra_bytes(d, n);
 }
 
 // partial[z][i][j] = sum_{k in slice z} X[i][k] X[j][k]   for tiles with bj <= bi
@@ -99,8 +101,10 @@ __global__ void __launch_bounds__(256) syrk_fp32_kernel(const float* __restrict_
 }
 
 // H[i][j] = H[j][i] = (accumulate ? H[i][j] : 0) + 2 * sum_z partial[z][i][j]     for j <= i
+// err (nullable): a non-zero flag from the producing kernel turns the whole result into NaN.
 __global__ void __launch_bounds__(256) hessian_finalize_kernel(const float* __restrict__ partial, int splits, int d,
-                                                               float* __restrict__ H, int ldh, int accumulate) {
+                                                               float* __restrict__ H, int ldh, int accumulate,
+                                                               const int* __restrict__ err) {
     const int i = blockIdx.y;
     const int j = blockIdx.x * 256 + threadIdx.x;
     if (j > i || j >= d) return;
@@ -108,14 +112,15 @@ __global__ void __launch_bounds__(256) hessian_finalize_kernel(const float* __re
     for (int z = 0; z < splits; ++z) s += partial[(size_t)z * d * d + (size_t)i * d + j];
     float v = 2.f * s;
     if (accumulate) v += H[(size_t)i * ldh + j];
+    if (err && *err != 0) v = __int_as_float(0x7fc00000);
     H[(size_t)i * ldh + j] = v;
     H[(size_t)j * ldh + i] = v;
 }
 
 obc_status hessian_finalize_launch(const float* partial, int splits, int d, float* H, int ldh, int accumulate,
-                                   cudaStream_t stream) {
+                                   const int* err, cudaStream_t stream) {
     dim3 grid((d + 255) / 256, d);
-    hessian_finalize_kernel<<<grid, 256, 0, stream>>>(partial, splits, d, H, ldh, accumulate);
+    hessian_finalize_kernel<<<grid, 256, 0, stream>>>(partial, splits, d, H, ldh, accumulate, err);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
@@ -132,7 +137,7 @@ obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, fl
     syrk_fp32_kernel<<<grid, 256, 0, stream>>>(X, d, n, ldx, slice, partial);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
-    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, stream);
+    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, nullptr, stream);
 }
 
 }  // namespace obc

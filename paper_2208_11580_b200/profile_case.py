@@ -1,4 +1,4 @@
-"""Small stand-alone run of the row elimination engine for profiler captures.
+"""Small stand-alone run of the row elimination engine (or the Hessian kernel) for profiler captures.
 
   python -m paper_2208_11580_b200.profile_case --d 1152 --rows 148 --mode prune --repeat 2
 
@@ -24,7 +24,8 @@ def main():
     ap.add_argument("--d", type=int, default=1152)
     ap.add_argument("--rows", type=int, default=148)
     ap.add_argument("--n", type=int, default=0)
-    ap.add_argument("--mode", default="prune", choices=["prune", "quant"])
+    ap.add_argument("--mode", default="prune", choices=["prune", "quant", "hessian"])
+    ap.add_argument("--prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
     ap.add_argument("--repeat", type=int, default=2)
     a = ap.parse_args()
     d, R = a.d, a.rows
@@ -32,6 +33,20 @@ def main():
     W, X = obc_synth.make_small(R, d, n, 4242, "relu")
     Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
     H = torch.empty(d, d, dtype=torch.float32, device="cuda")
+    if a.mode == "hessian":
+        prec = {"fp32": obc.PREC_FP32, "tf32": obc.PREC_TF32, "bf16x3": obc.PREC_BF16X3}[a.prec]
+        ws = torch.empty(obc.obc_workspace_bytes(obc.OP_HESSIAN, 0, d, n), dtype=torch.uint8, device="cuda")
+        times = []
+        for _ in range(a.repeat):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            obc.obc_hessian(Xd, H, prec=prec, ws=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        print(json.dumps({"d": d, "n": n, "mode": "hessian", "prec": a.prec, "ms": [round(t, 3) for t in times],
+                          "dense_equiv_TFLOPs": round(2.0 * d * d * n / (min(times) * 1e-3) / 1e12, 1)}))
+        return
     obc.obc_hessian(Xd, H)
     Hinv, info = obc.obc_hessian_inverse(H, obc_synth.DAMP_REL)
     order = torch.zeros(R, d, dtype=torch.int32, device="cuda")

@@ -54,8 +54,11 @@ def run_trace(obc, Wd, Hinv, steps=None, want_trace=False, row_begin=0, row_coun
 
 
 # ---------------------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("prec", [0])
-@pytest.mark.parametrize("d,n", [(64, 1024), (5, 37), (130, 4100), (576, 2048)])
+HESSIAN_TOL = {0: 2e-5, 1: 2e-3, 2: 3e-5}     # FP32 CUDA cores, TF32 and BF16x3 tensor cores; relative to max|H|
+
+
+@pytest.mark.parametrize("prec", [0, 1, 2])
+@pytest.mark.parametrize("d,n", [(64, 1024), (5, 37), (130, 4100), (576, 2048), (300, 20000)])
 def test_hessian_matches_fp64(obc, d, n, prec):
     _, X = obc_synth.make_small(1, d, n, 100 + d)
     ldx = (n + 3) // 4 * 4
@@ -66,13 +69,15 @@ def test_hessian_matches_fp64(obc, d, n, prec):
     ref = oracle.hessian(X)
     got = H.cpu().numpy().astype(np.float64)
     assert np.array_equal(got, got.T)
-    assert np.abs(got - ref).max() <= 2e-5 * np.abs(ref).max()
+    tol = HESSIAN_TOL[prec]
+    print("hessian", d, n, prec, np.abs(got - ref).max() / np.abs(ref).max())
+    assert np.abs(got - ref).max() <= tol * np.abs(ref).max()
     # accumulation over chunks of the calibration axis
     H2 = torch.zeros(d, ldh, dtype=torch.float32, device="cuda")[:, :d]
     h = (n // 2 + 3) // 4 * 4
     obc.obc_hessian(Xd[:, :h], H2, accumulate=False, prec=prec)
     obc.obc_hessian(Xd[:, h:], H2, accumulate=True, prec=prec)
-    assert np.abs(H2.cpu().numpy() - ref).max() <= 2e-5 * np.abs(ref).max()
+    assert np.abs(H2.cpu().numpy() - ref).max() <= tol * np.abs(ref).max()
 
 
 @pytest.mark.parametrize("d", [5, 48, 64, 100, 576, 1000])
