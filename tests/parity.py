@@ -29,6 +29,14 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
     assert np.all(res["status"] == 0), f"oracle rejected the GPU order: {res['status']}"
     differ = res["best"] != gpu_order
     gap = res["forced_gap"]
+    if mode == "quant":
+        # OBQ scores are squared DIFFERENCES w - q(w) over the pivot diagonal, so their natural scale is the score
+        # of a half-step error at that pivot, (Delta/2)^2/[Hinv]_pp; the margin is taken relative to
+        # max(score, that scale): a tiny score is only known to the absolute accuracy of w.
+        half = 0.5 * np.broadcast_to(np.asarray(scale, dtype=np.float64), (rows,))[:, None]
+        s_f = res["loss"]
+        s_ref = np.maximum(s_f, half * half / np.maximum(res["pivot_diag"], 1e-300))
+        gap = gap * s_f / np.maximum(s_ref, 1e-300)
     bad = differ & (gap > MARGIN_TOL)
     stats = dict(steps=int(rows * steps), picks_differ=int(differ.sum()), max_gap_at_differ=float(gap[differ].max()) if differ.any() else 0.0,
                  sub_1e5_margin=int((res["margin"] < 1e-5).sum()))
