@@ -60,6 +60,14 @@ typedef enum {
     OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5
 } obc_op;
 
+/* Which row elimination engine obc_prune_trace / obc_prune_apply / obc_quantize run (all compute Algorithm 1 /
+ * Algorithm 3; they differ in how the Lemma-1 updates reach the row's private inverse Hessian):
+ *   STREAMING  one pass over the row's active triangle per step (rank-1 update, bound by memory bandwidth);
+ *   BLOCKED    the updates are held back as vectors and applied several at a time, so the triangle is read and
+ *              written once per block of steps; the pivot column of a step is corrected by the pending vectors;
+ *   AUTO       = BLOCKED. */
+typedef enum { OBC_ENGINE_AUTO = 0, OBC_ENGINE_STREAMING = 1, OBC_ENGINE_BLOCKED = 2 } obc_engine;
+
 #define OBC_MAX_DCOL 5120      /* per-row state of the elimination engine lives in one CTA's shared memory */
 
 typedef void *obc_stream;      /* a cudaStream_t (NULL = default stream) */
@@ -68,6 +76,13 @@ const char *obc_status_string(obc_status s);
 
 /* Diagnostic (host function): number of kernels this library has launched in the calling process so far. */
 unsigned long long obc_kernel_launches(void);
+
+/* Process-wide engine selection (host function; takes effect for calls made after it returns; not meant to be
+ * changed while another thread is inside a library call).  threads: threads per row of the BLOCKED engine
+ * (128, 256, 512; 0 = chosen from d_col).  max_pending: upper limit on the number of deferred updates
+ * (1..64; 0 = as many as the shared memory holds).  Workspace sizes reported by obc_workspace_bytes are valid
+ * for every choice.  Returns OBC_ERR_INVALID_ARG for values outside these sets. */
+obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
 
 /* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).
  * n is only used by OBC_OP_HESSIAN; row_count (the rows one call processes) by the three row-engine ops,

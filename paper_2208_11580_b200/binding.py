@@ -16,9 +16,10 @@ _LIBPATH = os.path.join(_HERE, "libobc.so")
 OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE = range(6)
 PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
 FLAG_OUTLIERS = 1
+ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
+    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -50,6 +51,8 @@ def load_library():
     lib.obc_status_string.argtypes = [c_int]
     lib.obc_kernel_launches.restype = ctypes.c_ulonglong
     lib.obc_kernel_launches.argtypes = []
+    lib.obc_set_engine.restype = c_int
+    lib.obc_set_engine.argtypes = [c_int, c_int, c_int]
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
@@ -80,6 +83,11 @@ def obc_status_string(status: int) -> str:
 
 def obc_kernel_launches() -> int:
     return int(load_library().obc_kernel_launches())
+
+
+def obc_set_engine(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0) -> None:
+    """Process-wide choice of the row elimination engine (streaming rank-1 passes or deferred block updates)."""
+    _raise(load_library().obc_set_engine(int(engine), int(threads), int(max_pending)), "obc_set_engine")
 
 
 def _ptr(t):

@@ -1,6 +1,6 @@
 // C ABI of the OBC library: argument checks on the host (nothing is launched or written when they fail),
 // then dispatch to the kernels.  See include/obc.h for the contract of every entry point.
-#include "common.cuh"
+#include "engine.cuh"
 #include <atomic>
 #include <mutex>
 
@@ -28,6 +28,11 @@ obc_status device_info(DeviceInfo* out) {
     *out = cache[dev];
     return OBC_OK;
 }
+
+static std::atomic<int> g_engine{OBC_ENGINE_AUTO}, g_engine_threads{0}, g_engine_pending{0};
+int engine_choice() { return g_engine.load(std::memory_order_relaxed); }
+int engine_threads_choice() { return g_engine_threads.load(std::memory_order_relaxed); }
+int engine_pending_choice() { return g_engine_pending.load(std::memory_order_relaxed); }
 
 static bool mat_ok(const void* p, int64_t ld, int64_t min_ld) { return p && ld >= min_ld; }
 static bool mat_aligned(const void* p, int64_t ld) { return aligned16(p) && (ld % 4 == 0); }
@@ -58,6 +63,17 @@ const char* obc_status_string(obc_status s) {
 }
 
 unsigned long long obc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+obc_status obc_set_engine(obc_engine engine, int threads, int max_pending) {
+    if (engine != OBC_ENGINE_AUTO && engine != OBC_ENGINE_STREAMING && engine != OBC_ENGINE_BLOCKED)
+        return OBC_ERR_INVALID_ARG;
+    if (threads != 0 && threads != 128 && threads != 256 && threads != 512) return OBC_ERR_INVALID_ARG;
+    if (max_pending < 0 || max_pending > 64) return OBC_ERR_INVALID_ARG;
+    g_engine.store((int)engine, std::memory_order_relaxed);
+    g_engine_threads.store(threads, std::memory_order_relaxed);
+    g_engine_pending.store(max_pending, std::memory_order_relaxed);
+    return OBC_OK;
+}
 
 size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
     if (d_col <= 0 || row_count < 0) return 0;

@@ -15,8 +15,7 @@
 // part strided) and the last active row  ->  update w, diag, u = v/dpp; move slot `last` into slot p
 // ->  stream the triangle once:  H[i][j] -= v[i]*u[j]  (128-bit loads/stores, one warp per matrix row).
 // Once m*m fits in shared memory the triangle is moved on chip and the row finishes there.
-#include "common.cuh"
-#include <math_constants.h>
+#include "engine.cuh"
 
 namespace obc {
 
@@ -24,46 +23,9 @@ constexpr int ENGINE_THREADS = 1024;
 constexpr int ENGINE_WARPS = ENGINE_THREADS / 32;
 constexpr int ENGINE_FIXED_SMEM = 1280;       // 1024 B reduction scratch + broadcast block
 
-enum EngineMode { MODE_PRUNE = 0, MODE_REPLAY = 1, MODE_QUANT = 2, MODE_REPLAY_QUANT = 3 };
-
-struct EngineArgs {
-    const float* W; int ldw;
-    int d; int row_begin; int row_count;
-    const float* Hinv; int ldhi;
-    int mode; int steps;
-    const int32_t* forced_order; const int32_t* forced_counts;
-    float* scale; float* zero; int bits; int symmetric; int flags;
-    int32_t* order; float* loss;
-    float* w_trace; int trace_steps;
-    float* W_out; int ldwo;
-    int32_t* codes; int32_t* row_status;
-    float* Hws; int ldp;                  // private triangles: gridDim.x blocks of d x ldp floats
-    int ms;                               // on-chip threshold: finish in shared memory once m <= ms
-    int cap;                              // d rounded up to a multiple of 4
-};
-
-struct Bcast {                            // block-wide broadcast values, written by one thread
-    double e, dpp, qp, code;
-    double sc, ze, mq;
-    int slot; int fail; int op; int pad_;
-};
-
 struct State {                            // views into shared memory (layout differs per phase)
     double* wd; double* dg; int* perm; float* v; float* u; float* lr;
 };
-
-__device__ __forceinline__ bool key_less(double s, int o, double s2, int o2) {
-    return s < s2 || (s == s2 && o < o2);
-}
-
-// q(x) on the uniform grid; all FP64 so that the integer code is decided in the same precision as the
-// FP64 reference decides it.
-__device__ __forceinline__ double grid_q(double x, double sc, double ze, double mq, double* code) {
-    double c = rint(x / sc) + ze;
-    c = fmin(fmax(c, 0.0), mq);
-    *code = c;
-    return sc * (c - ze);
-}
 
 // Block-wide argmin of (score, original index) over slots [0, m).  quant: score uses q(w)-w.
 // With outliers: any slot with |q(w)-w| > sc/2 wins by largest error (Section 4, "Quantization Outliers").
@@ -411,7 +373,7 @@ static int engine_pick_ms(int d, int cap, int smem_optin) {
     return ms;
 }
 
-size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
+size_t streaming_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
     const int cap = (d + 3) & ~3;
     const int ms = engine_pick_ms(d, cap, di.smem_optin);
     if (d <= ms) return 256;
@@ -420,7 +382,7 @@ size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
     return round_up((size_t)blocks * d * cap * sizeof(float), 256);
 }
 
-obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
+obc_status streaming_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
     DeviceInfo di;
     obc_status st = device_info(&di);
     if (st != OBC_OK) return st;
@@ -428,7 +390,7 @@ obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t s
     if (a.d > OBC_MAX_DCOL || engine_smem_bytes(a.cap, 2) > (size_t)di.smem_optin) return OBC_ERR_UNSUPPORTED;
     a.ms = engine_pick_ms(a.d, a.cap, di.smem_optin);
     int blocks = di.sm_count < a.row_count ? di.sm_count : a.row_count;
-    const size_t need = engine_workspace_bytes(a.row_count, a.d, di);
+    const size_t need = streaming_engine_workspace_bytes(a.row_count, a.d, di);
     if (!ws || !aligned256(ws) || ws_bytes < need) return OBC_ERR_WORKSPACE;
     a.Hws = reinterpret_cast<float*>(ws);
     a.ldp = a.cap;
@@ -438,6 +400,18 @@ obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t s
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
+}
+
+// ---- engine choice ----------------------------------------------------------------------------------------
+size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
+    const size_t s1 = streaming_engine_workspace_bytes(row_count, d, di);
+    const size_t s2 = blocked_engine_workspace_bytes(row_count, d, di);
+    return s1 > s2 ? s1 : s2;          // valid for either engine, whichever is selected at call time
+}
+
+static obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    if (engine_choice() == OBC_ENGINE_STREAMING) return streaming_engine_launch(a, ws, ws_bytes, stream);
+    return blocked_engine_launch(a, ws, ws_bytes, stream);
 }
 
 static EngineArgs base_args(const float* W, int ldw, int d_col, int row_begin, int row_count, const float* Hinv,

@@ -1,0 +1,616 @@
+// Row elimination engine with deferred Lemma-1 updates (Algorithm 1 / Algorithm 3 of "Optimal Brain
+// Compression"), one thread block per weight-matrix row, several rows per SM.
+//
+// A greedy step needs only three things from the row's inverse Hessian: its diagonal (for the scores), the
+// pivot column (for the weight update, Eq. 3 / Eq. 7) and, later, everything else.  Lemma 1 is a rank-1
+// update, so B of them can be held back as vectors z_b = H[:,p_b] / sqrt([H]_pp) (each taken from the matrix
+// as it would be at its own step) and applied together:
+//       H_true = H_stored - sum_b z_b z_b^T .
+// The pivot column of a step is then one column of H_stored corrected by the pending vectors (m x B work),
+// and the m x m matrix is read and written once per B steps instead of once per step.  Picks, weights and
+// losses are the same as with step-by-step updates up to the order of the FP32 roundings.
+//
+// Layout.  The private copy keeps the lower triangle only (the matrix stays symmetric).  Slots [0, m0) are
+// fixed between two flushes; eliminated slots are marked dead (perm = -1).  The flush applies the pending
+// vectors and compacts at the same time: a dead slot h below the new size m1 is taken over by a live slot
+// s >= m1, i.e. element (i, j) of the new triangle is read from (max(si, sj), min(si, sj)) of the old one.
+// All such foreign reads come from rows >= m1, which the flush never writes, so it runs in place.
+// The flush works on warp tiles of 8 rows x 128 columns with the 8 x 4 sub-tile of each lane in registers;
+// the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
+// the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
+// finishes on chip with step-by-step updates.
+#include "engine.cuh"
+
+namespace obc {
+
+constexpr int BLK_MAXB = 64;
+constexpr int BLK_OFF_BC = 1024;              // Bcast
+constexpr int BLK_OFF_PV = 1280;              // int pv[64]   slots eliminated since the last flush
+constexpr int BLK_OFF_HL = 1536;              // int hl[64]   holes (dead slots below the new size)
+constexpr int BLK_OFF_MV = 1792;              // int mv[64]   live slots that move into the holes
+constexpr int BLK_OFF_CM = 2048;              // uint32 colmask[160]: bit j set = column j is a hole
+constexpr int BLK_FIXED = 2048 + 640;
+
+__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull) {
+    return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0);
+}
+static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
+
+template <int NT>
+__device__ __forceinline__ void blk_reduce_pick(double bs, int bo, int bslot, double oe, int oo, int oslot,
+                                                bool outliers, Bcast* bc, char* scratch) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+        const double s2 = __shfl_xor_sync(0xffffffffu, bs, off);
+        const int o2 = __shfl_xor_sync(0xffffffffu, bo, off);
+        const int l2 = __shfl_xor_sync(0xffffffffu, bslot, off);
+        if (key_less(s2, o2, bs, bo)) { bs = s2; bo = o2; bslot = l2; }
+        if (outliers) {
+            const double e2 = __shfl_xor_sync(0xffffffffu, oe, off);
+            const int p2 = __shfl_xor_sync(0xffffffffu, oo, off);
+            const int q2 = __shfl_xor_sync(0xffffffffu, oslot, off);
+            if (e2 > oe || (e2 == oe && p2 < oo)) { oe = e2; oo = p2; oslot = q2; }
+        }
+    }
+    double* rs = reinterpret_cast<double*>(scratch);            // [32] scores
+    double* re = rs + 32;                                       // [32] outlier errors
+    int* ro = reinterpret_cast<int*>(re + 32);                  // [32] orig, [32] slot, [32] o-orig, [32] o-slot
+    if (lane == 0) {
+        rs[warp] = bs; ro[warp] = bo; ro[32 + warp] = bslot;
+        re[warp] = oe; ro[64 + warp] = oo; ro[96 + warp] = oslot;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const bool in = lane < NW;
+        bs = in ? rs[lane] : CUDART_INF; bo = in ? ro[lane] : 0x7fffffff; bslot = in ? ro[32 + lane] : -1;
+        oe = in ? re[lane] : -1.0; oo = in ? ro[64 + lane] : 0x7fffffff; oslot = in ? ro[96 + lane] : -1;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            const double s2 = __shfl_xor_sync(0xffffffffu, bs, off);
+            const int o2 = __shfl_xor_sync(0xffffffffu, bo, off);
+            const int l2 = __shfl_xor_sync(0xffffffffu, bslot, off);
+            if (key_less(s2, o2, bs, bo)) { bs = s2; bo = o2; bslot = l2; }
+            const double e2 = __shfl_xor_sync(0xffffffffu, oe, off);
+            const int p2 = __shfl_xor_sync(0xffffffffu, oo, off);
+            const int q2 = __shfl_xor_sync(0xffffffffu, oslot, off);
+            if (e2 > oe || (e2 == oe && p2 < oo)) { oe = e2; oo = p2; oslot = q2; }
+        }
+        if (lane == 0) bc->slot = (outliers && oslot >= 0) ? oslot : bslot;
+    }
+    __syncthreads();
+}
+
+// Block-wide argmin of (score, original index) over the live slots of [0, m0).  Every slot gets an FP32
+// estimate of its score first; only the slots within 1e-4 of the thread's best estimate are then scored
+// with the FP64 division, so the result (ties included) is the exact FP64 argmin.
+template <int NT, int KMAX>
+__device__ void blk_argmin(const double* wd, const double* dg, const int* perm, int m0, bool quant, bool outliers,
+                           Bcast* bc, char* scratch) {
+    const int tid = threadIdx.x;
+    const double sc = bc->sc, ze = bc->ze, mq = bc->mq;
+    float sa[KMAX];
+    float smin = CUDART_INF_F;
+    double oe = -1.0;
+    int oo = 0x7fffffff, oslot = -1;
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+        const int j = tid + k * NT;
+        sa[k] = CUDART_NAN_F;
+        if (j < m0 && perm[j] >= 0) {
+            const double w = wd[j];
+            double err = -w, code;
+            if (quant) err = grid_q(w, sc, ze, mq, &code) - w;
+            sa[k] = __double2float_rn(err * err) / __double2float_rn(dg[j]);
+            smin = fminf(smin, sa[k]);                       // fminf ignores a NaN estimate
+            if (outliers) {
+                const double a = fabs(err);
+                const int o = perm[j];
+                if (a > 0.5 * sc && (a > oe || (a == oe && o < oo))) { oe = a; oo = o; oslot = j; }
+            }
+        }
+    }
+    const float thr = smin + 1e-4f * fabsf(smin);
+    double bs = CUDART_INF;
+    int bo = 0x7fffffff, bslot = -1;
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+        const int j = tid + k * NT;
+        if (sa[k] <= thr || (sa[k] == smin)) {               // false for NaN estimates and for idle lanes
+            const double w = wd[j];
+            double err = -w, code;
+            if (quant) err = grid_q(w, sc, ze, mq, &code) - w;
+            const double s = err * err / dg[j];
+            const int o = perm[j];
+            if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
+        }
+    }
+    blk_reduce_pick<NT>(bs, bo, bslot, oe, oo, oslot, outliers, bc, scratch);
+}
+
+// Applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts
+// it to m1 rows.  srcm[i] = old slot whose data new slot i takes (i itself unless i is a hole).
+template <int NT>
+__device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m1, int nb, const float* Z, int ldz,
+                                          const unsigned short* srcm, const uint32_t* colmask) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nrg = (m1 + 7) >> 3;
+    for (int rg = warp; rg < nrg; rg += NW) {
+        const int i0 = rg << 3;
+        const int nrows = min(8, m1 - i0);
+        int sr[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) sr[r] = (r < nrows) ? (int)srcm[i0 + r] : i0;
+        const int jend = i0 + nrows;                           // columns [0, jend) hold data of this row group
+        for (int c0 = 0; c0 < jend; c0 += 128) {
+            const int j = c0 + (lane << 2);
+            if (j >= jend) continue;                           // whole float4 above the diagonal of every row
+            float4 acc[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < nrows && j <= i0 + r)
+                    acc[r] = *reinterpret_cast<const float4*>(Hp + (size_t)sr[r] * ldp + j);
+            }
+            // columns of this lane that are holes: their data sits in the mover's row
+            const uint32_t my4 = (colmask[j >> 5] >> (j & 31)) & 0xFu;
+            if (my4) {
+#pragma unroll
+                for (int comp = 0; comp < 4; ++comp) {
+                    if (!((my4 >> comp) & 1u)) continue;
+                    const int jj = j + comp;
+                    const int sj = (int)srcm[jj];
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        if (r < nrows && jj <= i0 + r) {
+                            const int hi = max(sr[r], sj), lo = min(sr[r], sj);
+                            const float val = Hp[(size_t)hi * ldp + lo];
+                            if (comp == 0) acc[r].x = val; else if (comp == 1) acc[r].y = val;
+                            else if (comp == 2) acc[r].z = val; else acc[r].w = val;
+                        }
+                    }
+                }
+            }
+            for (int b = 0; b < nb; ++b) {
+                const float* zb = Z + (size_t)b * ldz;
+                const float4 za = *reinterpret_cast<const float4*>(zb + i0);
+                const float4 zc = *reinterpret_cast<const float4*>(zb + i0 + 4);
+                const float4 zj = *reinterpret_cast<const float4*>(zb + j);
+                const float zi[8] = {za.x, za.y, za.z, za.w, zc.x, zc.y, zc.z, zc.w};
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    acc[r].x = fmaf(-zi[r], zj.x, acc[r].x);
+                    acc[r].y = fmaf(-zi[r], zj.y, acc[r].y);
+                    acc[r].z = fmaf(-zi[r], zj.z, acc[r].z);
+                    acc[r].w = fmaf(-zi[r], zj.w, acc[r].w);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+                if (r < nrows && j <= i0 + r)
+                    *reinterpret_cast<float4*>(Hp + (size_t)(i0 + r) * ldp + j) = acc[r];
+        }
+    }
+}
+
+// Step-by-step Lemma-1 update on the shared-memory triangle S (leading dimension lds) in the coordinates
+// that hold after slot `last` moved into slot pm (pm < 0: nothing moved); mp = rows left.
+template <int NT>
+__device__ __forceinline__ void blk_pass_shared(float* S, int lds, int mp, int pm, const float* v, const float* u,
+                                                const float* lr) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = warp; i < mp; i += NW) {
+        float* row = S + i * lds;
+        const float nv = -v[i];
+        for (int j = lane; j <= i; j += 32) {
+            const float base = (i == pm) ? lr[j] : (j == pm ? lr[i] : row[j]);
+            row[j] = fmaf(nv, u[j], base);
+        }
+    }
+}
+
+template <int NT, int KMAX>
+__global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
+    extern __shared__ __align__(16) char smem[];
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d = a.d, cap = a.cap, ms = a.ms;
+    char* scratch = smem;
+    Bcast* bc = reinterpret_cast<Bcast*>(smem + BLK_OFF_BC);
+    int* pv = reinterpret_cast<int*>(smem + BLK_OFF_PV);
+    int* hl = reinterpret_cast<int*>(smem + BLK_OFF_HL);
+    int* mv = reinterpret_cast<int*>(smem + BLK_OFF_MV);
+    uint32_t* colmask = reinterpret_cast<uint32_t*>(smem + BLK_OFF_CM);
+    double* wd = reinterpret_cast<double*>(smem + BLK_FIXED);
+    double* dg = wd + cap;
+    int* perm = reinterpret_cast<int*>(dg + cap);
+    unsigned short* srcm = reinterpret_cast<unsigned short*>(perm + cap);
+    const bool has_wfull = a.w_trace != nullptr;
+    float* wfull = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, false));
+    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull));
+    // tail views (step-by-step phase in shared memory) share the panel's space
+    const int msr = (ms + 3) & ~3;
+    float* tv = panel;
+    float* tu = tv + msr;
+    float* tlr = tu + msr;
+    float* S = tlr + msr;
+    const int lds = ms + 1;
+    float* Hp = a.Hws ? a.Hws + (size_t)blockIdx.x * d * a.ldp : nullptr;
+    const int ldp = a.ldp;
+
+    for (int rr = blockIdx.x; rr < a.row_count; rr += gridDim.x) {
+        const int r = a.row_begin + rr;
+        int n_forced = 0, n_free = 0;
+        bool quant = false;
+        if (a.mode == MODE_PRUNE) { n_free = a.steps; }
+        else if (a.mode == MODE_REPLAY) { n_forced = a.forced_counts[r]; }
+        else if (a.mode == MODE_QUANT) { n_free = d; quant = true; }
+        else { n_forced = a.forced_counts[r]; n_free = d - n_forced; quant = true; }
+        if (n_forced < 0) n_forced = 0;
+        if (n_forced > d) n_forced = d;
+        if (n_free > d - n_forced) n_free = d - n_forced;
+        const int total = n_forced + n_free;
+        const bool outliers = quant && (a.flags & OBC_FLAG_OUTLIERS);
+
+        // ---- row set-up ------------------------------------------------------------------------------
+        for (int j = tid; j < d; j += NT) {
+            const float w = a.W[(size_t)r * a.ldw + j];
+            wd[j] = (double)w;
+            dg[j] = (double)a.Hinv[(size_t)j * a.ldhi + j];
+            perm[j] = j;
+            srcm[j] = (unsigned short)j;
+            if (has_wfull) wfull[j] = w;
+            if (a.codes) a.codes[(size_t)r * d + j] = -1;
+        }
+        for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
+        if (tid == 0) {
+            bc->fail = 0;
+            bc->sc = 1.0; bc->ze = 0.0; bc->mq = 0.0;
+            if (a.mode == MODE_QUANT) {
+                bc->sc = (double)a.scale[r]; bc->ze = (double)a.zero[r];
+                bc->mq = (double)grid_maxq(a.bits, a.symmetric);
+            }
+            a.row_status[r] = 0;
+        }
+        if (a.w_trace)
+            for (int j = tid; j < d; j += NT)
+                a.w_trace[((size_t)r * (a.trace_steps + 1)) * d + j] = a.W[(size_t)r * a.ldw + j];
+        bool tail = false;
+        if (d > ms && total > 0) {
+            for (int i = warp; i < d; i += NW) {
+                const float4* s4 = reinterpret_cast<const float4*>(a.Hinv + (size_t)i * a.ldhi);
+                float4* d4 = reinterpret_cast<float4*>(Hp + (size_t)i * ldp);
+                const int n4 = (i >> 2) + 1;
+                for (int j4 = lane; j4 < n4; j4 += 32) d4[j4] = s4[j4];
+            }
+        }
+        __syncthreads();
+
+        int m0 = d;                      // slots in use (tail phase: number of live slots)
+        int nb = 0;                      // pending vectors
+        int ldz = (m0 + 7) & ~7;
+        int bcur = min(a.max_pending, a.panel_floats / ldz);
+        int s = 0;
+        for (; s < total; ++s) {
+            if (!tail) {
+                if (d > ms && nb > 0 && (nb == bcur || m0 - nb <= ms)) {
+                    // ---- flush: apply the pending vectors and compact to m1 slots ------------------------
+                    const int m1 = m0 - nb;
+                    if (tid == 0) {
+                        int nh = 0, sp = m1;
+                        for (int b = 0; b < nb; ++b) {
+                            const int h = pv[b];
+                            if (h < m1) {
+                                while (sp < m0 - 1 && perm[sp] < 0) ++sp;
+                                hl[nh] = h; mv[nh] = sp; ++sp; ++nh;
+                            }
+                        }
+                        bc->nh = nh;
+                    }
+                    __syncthreads();
+                    const int nh = bc->nh;
+                    for (int idx = tid; idx < nh * nb; idx += NT) {
+                        const int q = idx / nb, b = idx - q * nb;
+                        panel[(size_t)b * ldz + hl[q]] = panel[(size_t)b * ldz + mv[q]];
+                    }
+                    if (tid < nh) {
+                        const int h = hl[tid];
+                        srcm[h] = (unsigned short)mv[tid];
+                        atomicOr(&colmask[h >> 5], 1u << (h & 31));
+                    }
+                    __syncthreads();
+                    blk_flush<NT>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
+                    __syncthreads();
+                    if (tid < nh) {
+                        const int h = hl[tid], sv = mv[tid];
+                        wd[h] = wd[sv]; dg[h] = dg[sv]; perm[h] = perm[sv];
+                        srcm[h] = (unsigned short)h;
+                        colmask[h >> 5] = 0u;
+                    }
+                    m0 = m1; nb = 0;
+                    ldz = (m0 + 7) & ~7;
+                    bcur = min(a.max_pending, a.panel_floats / ldz);
+                    __syncthreads();
+                }
+                if (m0 <= ms) {
+                    // ---- move on chip: slots [0, m0) are all live here and the stored triangle is current
+                    const float* src = (d > ms) ? Hp : a.Hinv;
+                    const int sld = (d > ms) ? ldp : a.ldhi;
+                    for (int i = warp; i < m0; i += NW)
+                        for (int j = lane; j <= i; j += 32) S[i * lds + j] = src[(size_t)i * sld + j];
+                    tail = true;
+                    __syncthreads();
+                }
+            }
+            const bool forced = s < n_forced;
+            const bool q_now = quant && !forced;
+            // ---- grid of the compound path: built from the survivors when the replay is over -----------
+            if (a.mode == MODE_REPLAY_QUANT && s == n_forced) {
+                float lo = 0.f, hi = 0.f;
+                for (int j = tid; j < m0; j += NT)
+                    if (perm[j] >= 0) { const float w = (float)wd[j]; lo = fminf(lo, w); hi = fmaxf(hi, w); }
+#pragma unroll
+                for (int off = 16; off; off >>= 1) {
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
+                    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
+                }
+                float* rf = reinterpret_cast<float*>(scratch);
+                if (lane == 0) { rf[warp] = lo; rf[32 + warp] = hi; }
+                __syncthreads();
+                if (tid == 0) {
+                    for (int k = 0; k < NW; ++k) { lo = fminf(lo, rf[k]); hi = fmaxf(hi, rf[32 + k]); }
+                    float sc, ze;
+                    grid_from_range(lo, hi, a.bits, a.symmetric, &sc, &ze);
+                    a.scale[r] = sc; a.zero[r] = ze;
+                    bc->sc = (double)sc; bc->ze = (double)ze; bc->mq = (double)grid_maxq(a.bits, a.symmetric);
+                }
+                __syncthreads();
+            }
+            // ---- pick the slot -------------------------------------------------------------------------
+            if (forced) {
+                if (tid == 0) bc->slot = -1;
+                __syncthreads();
+                const int f = a.forced_order[(size_t)r * d + s];
+                for (int j = tid; j < m0; j += NT)
+                    if (perm[j] == f) bc->slot = j;
+                __syncthreads();
+            } else {
+                blk_argmin<NT, KMAX>(wd, dg, perm, m0, q_now, outliers, bc, scratch);
+            }
+            const int p = bc->slot;
+            if (tid == 0) {
+                int fail = 0;
+                double dpp = 0, e = 0, qp = 0, code = -1;
+                if (p < 0) fail = 1;
+                else {
+                    bc->op = perm[p];
+                    dpp = dg[p];
+                    if (!(dpp > 0.0) || !isfinite(dpp) || !isfinite(wd[p])) fail = 1;
+                    else {
+                        if (q_now) qp = grid_q(wd[p], bc->sc, bc->ze, bc->mq, &code);
+                        e = wd[p] - qp;
+                    }
+                }
+                bc->fail = fail; bc->dpp = dpp; bc->e = e; bc->qp = qp; bc->code = code;
+            }
+            if (!tail) {
+                // ======================= deferred-update step ==============================================
+                float* zb = panel + (size_t)nb * ldz;
+                if (p >= 0) {
+                    // pivot column of the stored matrix, corrected by the pending vectors
+                    float c[KMAX], corr[KMAX];
+                    const float* rowp = Hp + (size_t)p * ldp;
+#pragma unroll
+                    for (int k = 0; k < KMAX; ++k) {
+                        const int j = tid + k * NT;
+                        c[k] = 0.f; corr[k] = 0.f;
+                        if (j < m0 && perm[j] >= 0) c[k] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                    }
+                    for (int b = 0; b < nb; ++b) {
+                        const float* zo = panel + (size_t)b * ldz;
+                        const float zp = zo[p];
+#pragma unroll
+                        for (int k = 0; k < KMAX; ++k) {
+                            const int j = tid + k * NT;
+                            if (j < m0) corr[k] = fmaf(zo[j], zp, corr[k]);
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < KMAX; ++k) {
+                        const int j = tid + k * NT;
+                        if (j < m0) zb[j] = (perm[j] >= 0) ? c[k] - corr[k] : 0.f;
+                    }
+                }
+                __syncthreads();
+                if (bc->fail) break;
+                {
+                    const double dpp = bc->dpp, f = bc->e / dpp, idpp = 1.0 / dpp;
+                    const float rs = (float)(1.0 / sqrt(dpp));
+                    const int op = bc->op;
+#pragma unroll
+                    for (int k = 0; k < KMAX; ++k) {
+                        const int j = tid + k * NT;
+                        if (j >= m0 || perm[j] < 0) continue;
+                        if (j == p) { zb[j] = 0.f; perm[j] = -1; continue; }
+                        const float vj = zb[j];
+                        const double nw = wd[j] - f * (double)vj;
+                        wd[j] = nw;
+                        dg[j] -= (double)vj * (double)vj * idpp;
+                        zb[j] = vj * rs;
+                        if (has_wfull) wfull[perm[j]] = (float)nw;
+                    }
+                    if (tid == 0) {
+                        pv[nb] = p;
+                        if (has_wfull) wfull[op] = (float)bc->qp;
+                        if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)bc->qp;
+                        if (!forced) {
+                            const int t = s - n_forced;
+                            if (a.order) a.order[(size_t)r * d + t] = op;
+                            if (a.loss) a.loss[(size_t)r * d + t] = (float)(bc->e * bc->e / dpp);
+                        }
+                        if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)bc->code;
+                    }
+                }
+                ++nb;
+                __syncthreads();
+                if (a.w_trace && s < a.trace_steps)
+                    for (int j = tid; j < d; j += NT)
+                        a.w_trace[((size_t)r * (a.trace_steps + 1) + s + 1) * d + j] = wfull[j];
+            } else {
+                // ======================= on-chip step (compaction at every step) ===========================
+                const int m = m0, last = m0 - 1;
+                if (p >= 0)
+                    for (int j = tid; j < m; j += NT) {
+                        tv[j] = (j <= p) ? S[p * lds + j] : S[j * lds + p];
+                        tlr[j] = S[last * lds + j];
+                    }
+                __syncthreads();
+                if (bc->fail) break;
+                {
+                    const double dpp = bc->dpp, f = bc->e / dpp;
+                    const int op = bc->op;
+                    for (int j = tid; j < m; j += NT) {
+                        if (j == p) continue;
+                        const float vj = tv[j];
+                        const double nw = wd[j] - f * (double)vj;
+                        const double nd = dg[j] - (double)vj * (double)vj / dpp;
+                        const float uj = (float)((double)vj / dpp);
+                        const int oj = perm[j];
+                        if (has_wfull) wfull[oj] = (float)nw;
+                        const int dst = (j == last) ? p : j;       // p != last here
+                        wd[dst] = nw; dg[dst] = nd; tu[dst] = uj;
+                        if (j == last) { perm[p] = oj; tv[p] = vj; tlr[p] = tlr[last]; }
+                    }
+                    if (tid == 0) {
+                        if (has_wfull) wfull[op] = (float)bc->qp;
+                        if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)bc->qp;
+                        if (!forced) {
+                            const int t = s - n_forced;
+                            if (a.order) a.order[(size_t)r * d + t] = op;
+                            if (a.loss) a.loss[(size_t)r * d + t] = (float)(bc->e * bc->e / dpp);
+                        }
+                        if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)bc->code;
+                    }
+                }
+                __syncthreads();
+                if (a.w_trace && s < a.trace_steps)
+                    for (int j = tid; j < d; j += NT)
+                        a.w_trace[((size_t)r * (a.trace_steps + 1) + s + 1) * d + j] = wfull[j];
+                const int pm = (p == last) ? -1 : p;
+                if (s + 1 < total) blk_pass_shared<NT>(S, lds, m - 1, pm, tv, tu, tlr);
+                --m0;
+                __syncthreads();
+            }
+        }
+        // ---- row epilogue ---------------------------------------------------------------------------------
+        if (s < total) {        // stopped early: report the step, mark what was not produced
+            if (tid == 0) a.row_status[r] = 1 + s;
+            const int t0 = (s < n_forced) ? 0 : s - n_forced;
+            for (int t = t0 + tid; t < n_free; t += NT) {
+                if (a.order) a.order[(size_t)r * d + t] = -1;
+                if (a.loss) a.loss[(size_t)r * d + t] = CUDART_INF_F;
+            }
+        }
+        if (a.W_out)            // eliminated entries were written at their step; the live ones follow here
+            for (int j = tid; j < m0; j += NT)
+                if (perm[j] >= 0) a.W_out[(size_t)r * a.ldwo + perm[j]] = (float)wd[j];
+        __syncthreads();
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------
+struct BlkPlan {
+    int nt;            // threads per block
+    int per_sm;        // blocks per SM the shared-memory split is made for
+    size_t smem;       // dynamic shared memory per block
+    int panel_floats;
+    int ms;
+};
+
+static int blk_pick_ms(int d, size_t panel_bytes) {
+    int ms = d < 1024 ? d : 1024;
+    if (ms < 2) ms = 2;
+    while (ms > 2 && blk_tail_bytes(ms) > panel_bytes) --ms;
+    return ms;
+}
+
+// Threads per block and blocks per SM by row length: short rows are bound by the latency of a step, so
+// several of them share an SM; long rows need the shared memory for pending vectors.
+static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out) {
+    const int cap = (d + 3) & ~3;
+    int nt = engine_threads_choice();
+    if (nt != 128 && nt != 256 && nt != 512) nt = d <= 1024 ? 128 : (d <= 2048 ? 256 : 512);
+    if (nt == 128 && cap > 1024) nt = 256;
+    if (nt == 256 && cap > 2048) nt = 512;
+    BlkPlan p;
+    p.nt = nt;
+    p.per_sm = 512 / nt;
+    // 1 KB per resident block is reserved by the hardware; keep every block's share 128-byte aligned
+    const size_t sm_total = (size_t)di.smem_optin + 1024;
+    size_t share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
+    if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
+    const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull);
+    const size_t min_panel = (size_t)4 * ((cap + 7) & ~7);
+    while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
+        p.per_sm >>= 1;
+        share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
+        if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
+    }
+    if (share < fixed + min_panel || share < fixed + blk_tail_bytes(2)) return false;
+    p.smem = share;
+    p.panel_floats = (int)((share - fixed) / 4);
+    p.ms = blk_pick_ms(d, share - fixed);
+    *out = p;
+    return true;
+}
+
+size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
+    BlkPlan p;
+    if (!blk_plan(d, true, di, &p)) return 256;
+    if (d <= p.ms) return 256;
+    const int cap = (d + 3) & ~3;
+    int blocks = di.sm_count * 4;                 // the largest grid any thread-count choice uses
+    if (row_count > 0 && row_count < blocks) blocks = row_count;
+    return round_up((size_t)blocks * d * cap * sizeof(float), 256);
+}
+
+template <int NT, int KMAX>
+static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
+    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)smem));
+    blocked_engine_kernel<NT, KMAX><<<blocks, NT, smem, stream>>>(a);
+    count_launch();
+    OBC_CUDA_TRY(cudaGetLastError());
+    return OBC_OK;
+}
+
+obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    DeviceInfo di;
+    obc_status st = device_info(&di);
+    if (st != OBC_OK) return st;
+    a.cap = (a.d + 3) & ~3;
+    if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    BlkPlan p;
+    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p)) return OBC_ERR_UNSUPPORTED;
+    a.ms = p.ms;
+    a.panel_floats = p.panel_floats;
+    int mp = engine_pending_choice();
+    a.max_pending = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB;
+    int blocks = di.sm_count * p.per_sm;
+    if (a.row_count < blocks) blocks = a.row_count;
+    a.Hws = nullptr;
+    a.ldp = a.cap;
+    if (a.d > p.ms) {
+        const size_t need = round_up((size_t)blocks * a.d * a.cap * sizeof(float), 256);
+        if (!ws || !aligned256(ws) || ws_bytes < need) return OBC_ERR_WORKSPACE;
+        a.Hws = reinterpret_cast<float*>(ws);
+    }
+    if (p.nt == 128) return blk_launch<128, 8>(a, blocks, p.smem, stream);
+    if (p.nt == 256) return blk_launch<256, 8>(a, blocks, p.smem, stream);
+    return blk_launch<512, 10>(a, blocks, p.smem, stream);
+}
+
+}  // namespace obc

@@ -27,8 +27,13 @@ def main():
     ap.add_argument("--mode", default="prune", choices=["prune", "quant", "hessian"])
     ap.add_argument("--prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
     ap.add_argument("--repeat", type=int, default=2)
+    ap.add_argument("--engine", default="auto", choices=["auto", "streaming", "blocked"])
+    ap.add_argument("--threads", type=int, default=0, help="blocked engine: threads per row (0 = from d)")
+    ap.add_argument("--pending", type=int, default=0, help="blocked engine: limit on deferred updates (0 = max)")
     a = ap.parse_args()
     d, R = a.d, a.rows
+    obc.obc_set_engine({"auto": obc.ENGINE_AUTO, "streaming": obc.ENGINE_STREAMING, "blocked": obc.ENGINE_BLOCKED}[a.engine],
+                       a.threads, a.pending)
     n = a.n or 2 * d
     W, X = obc_synth.make_small(R, d, n, 4242, "relu")
     Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
@@ -73,7 +78,7 @@ def main():
     assert int(info.item()) == 0 and int(status.abs().sum()) == 0
     m = np.arange(1, d + 1, dtype=np.float64)
     nbytes = R * float((8 * m * m).sum())
-    print(json.dumps({"d": d, "rows": R, "mode": a.mode, "ms": [round(t, 3) for t in times],
+    print(json.dumps({"d": d, "rows": R, "mode": a.mode, "engine": a.engine, "threads": a.threads, "pending": a.pending, "ms": [round(t, 3) for t in times],
                       "algorithmic_GBps": round(nbytes / (min(times) * 1e-3) / 1e9, 1),
                       "private_copies_MB": round(min(R, 148) * d * d * 4 / 1e6, 1)}))
 

@@ -13,11 +13,14 @@ pytestmark = pytest.mark.gpu
 DAMP = obc_synth.DAMP_REL
 
 
-@pytest.fixture(scope="module")
-def obc():
+@pytest.fixture(scope="module", params=["blocked", "streaming"])
+def obc(request):
+    """the library with one of its two row elimination engines selected; every test runs with both"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    return m
+    m.obc_set_engine(m.ENGINE_BLOCKED if request.param == "blocked" else m.ENGINE_STREAMING)
+    yield m
+    m.obc_set_engine(m.ENGINE_AUTO)
 
 
 def _sample(R, k, seed):

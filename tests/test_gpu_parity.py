@@ -11,11 +11,14 @@ pytestmark = pytest.mark.gpu
 DAMP = obc_synth.DAMP_REL
 
 
-@pytest.fixture(scope="module")
-def obc():
+@pytest.fixture(scope="module", params=["blocked", "streaming"])
+def obc(request):
+    """the library with one of its two row elimination engines selected; every test runs with both"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    return m
+    m.obc_set_engine(m.ENGINE_BLOCKED if request.param == "blocked" else m.ENGINE_STREAMING)
+    yield m
+    m.obc_set_engine(m.ENGINE_AUTO)
 
 
 def dev(a, dtype=None):
@@ -324,3 +327,38 @@ def test_nonfinite_rows_are_reported_not_trapped(obc):
     o = order.cpu().numpy()
     assert np.all(o[1, s[1] - 1:] == -1) and np.all(np.isinf(loss.cpu().numpy()[1, s[1] - 1:]))
     check_rows(Hinv.cpu().numpy(), W[[0, 2]], o[[0, 2]], loss.cpu().numpy()[[0, 2]])
+
+
+@pytest.mark.parametrize("threads,max_pending", [(128, 1), (128, 3), (256, 7), (512, 2), (512, 64), (0, 0)])
+@pytest.mark.parametrize("d,rows", [(9, 3), (301, 4), (640, 3)])
+def test_blocked_engine_block_sizes(threads, max_pending, d, rows):
+    """deferred-update engine: every thread count, block lengths from 1 (a flush per step) to the maximum, sizes
+    around the on-chip threshold; prune trace with the full weight trace, and OBQ"""
+    import paper_2208_11580_b200 as m
+    m.load_library()
+    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
+    try:
+        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 900 + d, "relu")
+        H = oracle.hessian(X).astype(np.float32)
+        ld = (d + 3) // 4 * 4
+        Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
+        Wd = padded(W, ld)
+        order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
+        assert int(status.abs().sum()) == 0
+        check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
+        scale = torch.zeros(rows, dtype=torch.float32, device="cuda")
+        zero = torch.zeros(rows, dtype=torch.float32, device="cuda")
+        maxq = m.obc_minmax_grid(Wd, 4, False, scale, zero)
+        Wq = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        codes = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
+        ql = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        qo = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
+        rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
+        m.obc_quantize(Wd, Hinv, scale, zero, 4, False, Wq, codes, rs, loss=ql, qorder=qo)
+        torch.cuda.synchronize()
+        assert int(rs.abs().sum()) == 0
+        check_rows(Hinv.cpu().numpy(), W, qo.cpu().numpy(), ql.cpu().numpy(), gpu_w=Wq.cpu().numpy(), mode="quant",
+                   scale=scale.cpu().numpy().astype(np.float64), zero=zero.cpu().numpy().astype(np.float64), maxq=maxq,
+                   gpu_codes=codes.cpu().numpy())
+    finally:
+        m.obc_set_engine(m.ENGINE_AUTO)
