@@ -6,10 +6,12 @@ One "step" is one pass of the whole hot path over one layer, through the C ABI:
   final weights (per configuration; see WORKLOADS).
 Prints ONE JSON line.  `value` = eliminated (pruned or quantised) weights per second over the whole job with
 inputs resident in HBM; `e2e` = the same with host<->device copies inside the timed region;
-`roofline` = achieved algorithmic GB/s of the elimination kernel against the measured HBM copy rate;
+`roofline` = bytes the elimination kernel has to move per launch over its CUDA-event time, against the measured
+HBM copy rate (for the blocked engine: one read + one write of the active triangle per block of deferred updates;
+the 8 m^2-per-step model of the step-by-step method is reported beside it);
 `cpu_baseline` = the FP64 oracle on a bounded sample of the same rows on this machine's host cores.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1..C5] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1..C5] [--engine blocked|streaming] [--impl reference]
 """
 from __future__ import annotations
 
@@ -44,6 +46,40 @@ def model_bytes_full(d: int, first: int | None = None, steps: int | None = None)
     steps = first if steps is None else steps
     m = np.arange(first, first - steps, -1, dtype=np.float64)
     return int((8.0 * m * m).sum())
+
+
+def blocked_schedule(plan: dict, first: int, steps: int):
+    """(m_after_flush, updates_applied) for every pass the blocked engine makes over a row's matrix when `steps`
+    eliminations start at active size `first`: it defers min(max_pending, panel_floats // round_up(m, 8)) updates,
+    flushes early when the live size reaches the on-chip threshold, and finishes in shared memory below it."""
+    ms, panel, maxp = plan["on_chip_below"], plan["panel_floats"], plan["max_pending"]
+    out, m0, left = [], first, steps
+    if first <= ms:
+        return out
+    while left > 0 and m0 > ms:
+        b = max(1, min(maxp, panel // ((m0 + 7) // 8 * 8)))
+        nb = min(b, m0 - ms, left)
+        left -= nb
+        if left <= 0:
+            break                      # the last block of a row is never written back
+        m0 -= nb
+        out.append((m0, nb))
+    return out
+
+
+def blocked_bytes_flops(plan: dict, d: int, first: int | None = None, steps: int | None = None):
+    """Bytes and flops one row of the blocked engine has to move / execute: the private lower triangle written once,
+    then per pass one read and one write of the compacted triangle (4 bytes per element) and 2 flops per element
+    and deferred update."""
+    first = d if first is None else first
+    steps = first if steps is None else steps
+    nbytes = 4.0 * d * (d + 1) / 2 if d > plan["on_chip_below"] else 0.0
+    flops = 0.0
+    for m1, nb in blocked_schedule(plan, first, steps):
+        tri = m1 * (m1 + 1) / 2
+        nbytes += 8.0 * tri
+        flops += 2.0 * tri * nb
+    return nbytes, flops
 
 
 def peaks():
@@ -142,7 +178,8 @@ class Layer:
         self.ws = t.empty(need, dtype=t.uint8, device=dev)
         self.W.copy_(t.from_numpy(W))
         self.X.copy_(t.from_numpy(X))
-        self.engine_ms = []          # (label, CUDA-event ms, algorithmic bytes) per engine launch since reset_timers()
+        self.engine_ms = []          # (label, CUDA-event ms, launch info) per engine launch since reset_timers()
+        self._info = {}
         self._pending = []
         self.eliminated = R * d * (2 if task == "prune+quant" else 1)
 
@@ -159,9 +196,10 @@ class Layer:
         o, R, d, task = self.obc, self.R, self.d, self.spec.task
         self._timed("hessian", 0, lambda: o.obc_hessian(self.X, self.H, prec=self.prec, ws=self.ws))
         self._timed("inverse", 0, lambda: o.obc_hessian_inverse(self.H, obc_synth.DAMP_REL, Hinv=self.Hinv, info=self.info, ws=self.ws))
-        full = R * model_bytes_full(d)
+        full = self.launch_info(with_trace=False)
         if task in ("prune", "prune+quant", "compound"):
-            self._timed("engine:prune_trace", full, lambda: o.obc_prune_trace(self.W, self.Hinv, self.order, self.loss, self.status,
+            full_t = self.launch_info(with_trace=self.trace is not None)
+            self._timed("engine:prune_trace", full_t, lambda: o.obc_prune_trace(self.W, self.Hinv, self.order, self.loss, self.status,
                                                                               w_trace=self.trace, ws=self.ws))
             for i, k in enumerate(self.ks):
                 self._timed("select", 0, lambda i=i, k=k: o.obc_select_global_mask(self.loss, self.order, k, self.counts[i], self.masks[i], ws=self.ws))
@@ -177,6 +215,22 @@ class Layer:
             self._timed("engine:replay_quantize", full, lambda: o.obc_quantize(
                 self.W, self.Hinv, self.scale, self.zero, self.spec.bits, self.spec.symmetric, self.Wq, self.codes, self.status,
                 prune_order=self.order, prune_counts=self.counts[0], ws=self.ws))
+
+    def launch_info(self, with_trace: bool):
+        """What one engine launch over all rows (every active size d..1 once per row) has to move and compute."""
+        R, d = self.R, self.d
+        key = bool(with_trace)
+        if key not in self._info:
+            plan = self.obc.obc_engine_plan(d, with_trace)
+            info = {"model_bytes": R * model_bytes_full(d), "plan": plan}
+            if plan["engine"] == self.obc.ENGINE_BLOCKED:
+                b, f = blocked_bytes_flops(plan, d)
+                info["own_bytes"], info["flops"] = R * b, R * f
+            else:   # streaming: one read + one write of the active lower triangle per step
+                m = np.arange(1, d + 1, dtype=np.float64)
+                info["own_bytes"], info["flops"] = R * float((4.0 * m * (m + 1)).sum()), R * float((m * (m + 1)).sum())
+            self._info[key] = info
+        return self._info[key]
 
     def reset_timers(self):
         self._pending = []
@@ -221,6 +275,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     obc.load_library()
+    obc.obc_set_engine(obc.ENGINE_BLOCKED if args.engine == "blocked" else obc.ENGINE_STREAMING)
     name = args.workload
     W, X, spec = obc_synth.make_layer(name)          # every rank compresses its own copy of the layer
     prec = {"fp32": obc.PREC_FP32, "tf32": obc.PREC_TF32, "bf16x3": obc.PREC_BF16X3}[args.hessian_prec]
@@ -295,24 +350,44 @@ def run_ours(args):
         return
     peak, peak_kind = peaks()
     eng_ms = sum(ms for _, ms, _ in engine_runs)
-    eng_bytes = sum(b for _, _, b in engine_runs)
     n_eng = max(1, len(engine_runs))
-    achieved = eng_bytes / (eng_ms * 1e-3) / 1e9 if eng_ms > 0 else 0.0
-    roofline = {"bound": "hbm", "kernel": "row_engine_kernel", "achieved": round(achieved, 1), "peak": peak,
-                "peak_kind": peak_kind, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "traffic": int(eng_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                "traffic_source": "scaled from the d=1152 x 148-row ncu capture by algorithmic bytes",
-                "algorithmic_bytes_per_launch": eng_bytes // n_eng, "ms_per_launch": round(eng_ms / n_eng, 3),
+    own_bytes = sum(i["own_bytes"] for _, _, i in engine_runs)
+    model_bytes = sum(i["model_bytes"] for _, _, i in engine_runs)
+    flops = sum(i["flops"] for _, _, i in engine_runs)
+    plan = engine_runs[0][2]["plan"] if engine_runs else obc.obc_engine_plan(layer.d)
+    blocked = plan["engine"] == obc.ENGINE_BLOCKED
+    sec = eng_ms * 1e-3
+    achieved = own_bytes / sec / 1e9 if sec > 0 else 0.0
+    fp32_peak = plan["sm_count"] * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12   # TFLOP/s, FMA = 2
+    roofline = {"bound": "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
+                "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": round(achieved / peak, 4),
+                "traffic": (None if blocked else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE)),
+                "traffic_source": ("see profiles/ for the ncu DRAM counters of this kernel on a smaller case" if blocked else
+                                   "scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
+                "algorithmic_bytes_per_launch": int(own_bytes // n_eng), "ms_per_launch": round(eng_ms / n_eng, 3),
                 "launches_timed": len(engine_runs),
-                "note": "algorithmic bytes = 8 m^2 per elimination step (full active block read+write); the kernel "
-                        "moves only the lower triangle (4 m^2), so frac can exceed 1 without re-use"}
+                "bytes_model": ("one write of the private lower triangle, then one read + one write of the compacted "
+                                "triangle per block of deferred updates" if blocked else
+                                "one read + one write of the active lower triangle per step"),
+                "step_by_step_model": {"bytes_per_launch": int(model_bytes // n_eng),
+                                       "GBps_equivalent": round(model_bytes / sec / 1e9, 1) if sec > 0 else 0.0,
+                                       "over_hbm_peak": round(model_bytes / sec / 1e9 / peak, 3) if sec > 0 else 0.0,
+                                       "note": "8 m^2 bytes per elimination step (read + write of the full active block), "
+                                               "the figure the step-by-step method has to move"},
+                "alu": {"achieved_tflops": round(flops / sec / 1e12, 2) if sec > 0 else 0.0, "fp32_peak_tflops": round(fp32_peak, 1),
+                        "frac": round(flops / sec / 1e12 / fp32_peak, 4) if sec > 0 else 0.0,
+                        "note": "2 flops per triangle element and update; peak = SMs x 128 FMA lanes x 2 x max SM clock"},
+                "plan": plan}
+    if blocked and args.compare_streaming:
+        roofline["streaming_engine"] = streaming_reference(layer, peak)
     cpu = cpu_baseline(name, W, layer.Hinv.cpu().numpy(), layer, args.cpu_seconds)
     out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
            "config": {"workload": f"{name}: {spec.note}", "d_row": layer.R, "d_col": layer.d, "n_calib": layer.n,
                       "task": spec.task, "bits": spec.bits, "sparsities": list(spec.sparsities),
-                      "hessian_prec": args.hessian_prec, "damp_rel": obc_synth.DAMP_REL,
+                      "hessian_prec": args.hessian_prec, "engine": args.engine, "damp_rel": obc_synth.DAMP_REL,
                       "l2": "per-row inverse-Hessian working set exceeds L2 (inputs larger than L2)"
                             if layer.R * layer.d * layer.d * 2 > 126e6 else "working set fits L2 (small case)",
                       "parallelism": f"rows of one layer per GPU; {world} independent layer(s)"},
@@ -324,6 +399,38 @@ def run_ours(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def streaming_reference(layer, peak):
+    """The step-by-step (streaming) engine on one wave of rows of the same layer, timed alone after the main
+    measurement: its achieved bytes per second against the HBM peak, for comparison with the blocked engine."""
+    import torch
+    obc = layer.obc
+    spec, d = layer.spec, layer.d
+    rows = min(layer.R, 148)
+    obc.obc_set_engine(obc.ENGINE_STREAMING)
+    try:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        def call():
+            if spec.task == "quant":
+                obc.obc_quantize(layer.W, layer.Hinv, layer.scale, layer.zero, spec.bits, spec.symmetric, layer.Wq, layer.codes,
+                                 layer.status, row_begin=0, row_count=rows, ws=layer.ws)
+            else:
+                obc.obc_prune_trace(layer.W, layer.Hinv, layer.order, layer.loss, layer.status, row_begin=0, row_count=rows, ws=layer.ws)
+        call()
+        torch.cuda.synchronize()
+        ev[0].record(); call(); ev[1].record()
+        torch.cuda.synchronize()
+        ms = ev[0].elapsed_time(ev[1])
+    finally:
+        obc.obc_set_engine(obc.ENGINE_BLOCKED)
+    m = np.arange(1, d + 1, dtype=np.float64)
+    tri = rows * float((4.0 * m * (m + 1)).sum())
+    model = rows * model_bytes_full(d)
+    return {"kernel": "row_engine_kernel", "rows": rows, "ms": round(ms, 3),
+            "triangle_GBps": round(tri / (ms * 1e-3) / 1e9, 1), "frac_of_peak": round(tri / (ms * 1e-3) / 1e9 / peak, 4),
+            "step_by_step_model_GBps": round(model / (ms * 1e-3) / 1e9, 1),
+            "note": "bytes = one read + one write of the active lower triangle per step"}
 
 
 def cpu_baseline(name, W, Hinv32, layer, budget_s):
@@ -396,6 +503,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--hessian-prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--engine", default="blocked", choices=["blocked", "streaming"],
+                    help="row elimination engine: deferred block updates (default) or one pass per step")
+    ap.add_argument("--no-compare-streaming", dest="compare_streaming", action="store_false",
+                    help="skip the extra timing of the streaming engine on one wave of rows")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -19,7 +19,7 @@ FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
+    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -53,6 +53,8 @@ def load_library():
     lib.obc_kernel_launches.argtypes = []
     lib.obc_set_engine.restype = c_int
     lib.obc_set_engine.argtypes = [c_int, c_int, c_int]
+    lib.obc_engine_plan.restype = c_int
+    lib.obc_engine_plan.argtypes = [c_int, c_int, ctypes.POINTER(ctypes.c_int32)]
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
@@ -88,6 +90,14 @@ def obc_kernel_launches() -> int:
 def obc_set_engine(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0) -> None:
     """Process-wide choice of the row elimination engine (streaming rank-1 passes or deferred block updates)."""
     _raise(load_library().obc_set_engine(int(engine), int(threads), int(max_pending)), "obc_set_engine")
+
+
+def obc_engine_plan(d_col: int, with_trace: bool = False) -> dict:
+    """How rows of length d_col would run on the current device under the present engine choice."""
+    plan = (ctypes.c_int32 * 8)()
+    _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), plan), "obc_engine_plan")
+    return {"engine": int(plan[0]), "threads": int(plan[1]), "rows_per_sm": int(plan[2]), "on_chip_below": int(plan[3]),
+            "panel_floats": int(plan[4]), "max_pending": int(plan[5]), "sm_count": int(plan[6])}
 
 
 def _ptr(t):

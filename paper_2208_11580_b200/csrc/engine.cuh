@@ -47,11 +47,26 @@ __device__ __forceinline__ double grid_q(double x, double sc, double ze, double 
     return sc * (c - ze);
 }
 
+// Same result as grid_q with one multiplication instead of the division wherever the product x * (1/sc) is
+// safely away from a rounding boundary (the two quotients differ by a few units in the last place at most);
+// next to a boundary the true quotient decides, as in grid_q.
+__device__ __forceinline__ double grid_q_fast(double x, double sc, double isc, double ze, double mq, double* code) {
+    const double t = x * isc;
+    double c = rint(t);
+    if (fabs(fabs(t - c) - 0.5) < 1e-9 * fmax(1.0, fabs(t))) c = rint(x / sc);
+    c = fmin(fmax(c + ze, 0.0), mq);
+    *code = c;
+    return sc * (c - ze);
+}
+
 // Launchers of the two engines (same arguments; each checks its own workspace need).
 size_t streaming_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di);
 size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di);
 obc_status streaming_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream);
 obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream);
+
+obc_status streaming_engine_plan(int d, int32_t* plan);
+obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan);
 
 // Process-wide engine choice (see obc_set_engine in obc.h).
 int engine_choice();

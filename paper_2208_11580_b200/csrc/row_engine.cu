@@ -402,6 +402,17 @@ obc_status streaming_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cuda
     return OBC_OK;
 }
 
+obc_status streaming_engine_plan(int d, int32_t* plan) {
+    DeviceInfo di;
+    obc_status st = device_info(&di);
+    if (st != OBC_OK) return st;
+    const int cap = (d + 3) & ~3;
+    if (d > OBC_MAX_DCOL || engine_smem_bytes(cap, 2) > (size_t)di.smem_optin) return OBC_ERR_UNSUPPORTED;
+    plan[0] = OBC_ENGINE_STREAMING; plan[1] = ENGINE_THREADS; plan[2] = 1; plan[3] = engine_pick_ms(d, cap, di.smem_optin);
+    plan[4] = 0; plan[5] = 1; plan[6] = di.sm_count; plan[7] = 0;
+    return OBC_OK;
+}
+
 // ---- engine choice ----------------------------------------------------------------------------------------
 size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
     const size_t s1 = streaming_engine_workspace_bytes(row_count, d, di);

@@ -19,77 +19,112 @@
 // the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
 // the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
 // finishes on chip with step-by-step updates.
+//
+// Step protocol.  Between two flushes slot j belongs to thread j mod NT, which is the only one to touch
+// wd[j], dg[j], perm[j] and its entries of the pending vectors.  Each thread proposes its best slot, the
+// warps combine the proposals and publish one record per warp (with the candidate's weight and diagonal),
+// and after the single barrier of the step every warp reads the records and derives the same winner, so
+// no second barrier is needed to announce it.  Records alternate between two buffers by step parity.
 #include "engine.cuh"
 
 namespace obc {
 
 constexpr int BLK_MAXB = 64;
-constexpr int BLK_OFF_BC = 1024;              // Bcast
-constexpr int BLK_OFF_PV = 1280;              // int pv[64]   slots eliminated since the last flush
-constexpr int BLK_OFF_HL = 1536;              // int hl[64]   holes (dead slots below the new size)
-constexpr int BLK_OFF_MV = 1792;              // int mv[64]   live slots that move into the holes
-constexpr int BLK_OFF_CM = 2048;              // uint32 colmask[160]: bit j set = column j is a hole
-constexpr int BLK_FIXED = 2048 + 640;
+constexpr int BLK_REC_BYTES = 640;            // one record buffer: 16 warps x (key, slot, orig, s, w, dg)
+constexpr int BLK_OFF_BC = 1280;              // Bcast (grid parameters, flush bookkeeping)
+constexpr int BLK_OFF_PV = 1536;              // int pv[64]   slots eliminated since the last flush
+constexpr int BLK_OFF_HL = 1792;              // int hl[64]   holes (dead slots below the new size)
+constexpr int BLK_OFF_MV = 2048;              // int mv[64]   live slots that move into the holes
+constexpr int BLK_OFF_CM = 2304;              // uint32 colmask[160]: bit j set = column j is a hole
+constexpr int BLK_OFF_RF = 2944;              // float rf[64]  min/max reduction of the compound grid
+constexpr int BLK_FIXED = 3200;
 
 __host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull) {
     return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0);
 }
 static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
 
-template <int NT>
-__device__ __forceinline__ void blk_reduce_pick(double bs, int bo, int bslot, double oe, int oo, int oslot,
-                                                bool outliers, Bcast* bc, char* scratch) {
-    constexpr int NW = NT / 32;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+struct Records {                              // views into one record buffer
+    unsigned* key; int* slot; int* orig; double* s; double* w; double* dgv;
+};
+__device__ __forceinline__ Records rec_view(char* scratch, int parity) {
+    char* b = scratch + parity * BLK_REC_BYTES;
+    Records r;
+    r.s = reinterpret_cast<double*>(b);       // [16]
+    r.w = r.s + 16;                           // [16]
+    r.dgv = r.w + 16;                         // [16]
+    r.key = reinterpret_cast<unsigned*>(r.dgv + 16);
+    r.slot = reinterpret_cast<int*>(r.key + 16);
+    r.orig = r.slot + 16;
+    return r;
+}
+
+// Monotone map of a float to an unsigned key (smaller float -> smaller key); NaN never reaches it.
+__device__ __forceinline__ unsigned float_key(float x) {
+    const unsigned u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+constexpr unsigned KEY_NONE = 0xFFFFFFFFu;
+
+struct Pick { int slot; int orig; double w; double dgv; };
+
+// Combines one candidate per lane into the lane holding the smallest (s, orig); key = float_key((float)s)
+// orders all but near-equal candidates, which are then compared exactly.  Returns the winning lane or -1.
+__device__ __forceinline__ int warp_winner(unsigned key, double s, int orig) {
+    const unsigned kmin = __reduce_min_sync(0xffffffffu, key);
+    if (kmin == KEY_NONE) return -1;
+    const unsigned cand = __ballot_sync(0xffffffffu, key == kmin);
+    if (__popc(cand) == 1) return __ffs(cand) - 1;
+    double bs = (key == kmin) ? s : CUDART_INF;
+    int bo = (key == kmin) ? orig : 0x7fffffff;
+    int bl = threadIdx.x & 31;
 #pragma unroll
     for (int off = 16; off; off >>= 1) {
         const double s2 = __shfl_xor_sync(0xffffffffu, bs, off);
         const int o2 = __shfl_xor_sync(0xffffffffu, bo, off);
-        const int l2 = __shfl_xor_sync(0xffffffffu, bslot, off);
-        if (key_less(s2, o2, bs, bo)) { bs = s2; bo = o2; bslot = l2; }
-        if (outliers) {
-            const double e2 = __shfl_xor_sync(0xffffffffu, oe, off);
-            const int p2 = __shfl_xor_sync(0xffffffffu, oo, off);
-            const int q2 = __shfl_xor_sync(0xffffffffu, oslot, off);
-            if (e2 > oe || (e2 == oe && p2 < oo)) { oe = e2; oo = p2; oslot = q2; }
-        }
+        const int l2 = __shfl_xor_sync(0xffffffffu, bl, off);
+        if (key_less(s2, o2, bs, bo)) { bs = s2; bo = o2; bl = l2; }
     }
-    double* rs = reinterpret_cast<double*>(scratch);            // [32] scores
-    double* re = rs + 32;                                       // [32] outlier errors
-    int* ro = reinterpret_cast<int*>(re + 32);                  // [32] orig, [32] slot, [32] o-orig, [32] o-slot
-    if (lane == 0) {
-        rs[warp] = bs; ro[warp] = bo; ro[32 + warp] = bslot;
-        re[warp] = oe; ro[64 + warp] = oo; ro[96 + warp] = oslot;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        const bool in = lane < NW;
-        bs = in ? rs[lane] : CUDART_INF; bo = in ? ro[lane] : 0x7fffffff; bslot = in ? ro[32 + lane] : -1;
-        oe = in ? re[lane] : -1.0; oo = in ? ro[64 + lane] : 0x7fffffff; oslot = in ? ro[96 + lane] : -1;
-#pragma unroll
-        for (int off = 16; off; off >>= 1) {
-            const double s2 = __shfl_xor_sync(0xffffffffu, bs, off);
-            const int o2 = __shfl_xor_sync(0xffffffffu, bo, off);
-            const int l2 = __shfl_xor_sync(0xffffffffu, bslot, off);
-            if (key_less(s2, o2, bs, bo)) { bs = s2; bo = o2; bslot = l2; }
-            const double e2 = __shfl_xor_sync(0xffffffffu, oe, off);
-            const int p2 = __shfl_xor_sync(0xffffffffu, oo, off);
-            const int q2 = __shfl_xor_sync(0xffffffffu, oslot, off);
-            if (e2 > oe || (e2 == oe && p2 < oo)) { oe = e2; oo = p2; oslot = q2; }
-        }
-        if (lane == 0) bc->slot = (outliers && oslot >= 0) ? oslot : bslot;
-    }
-    __syncthreads();
+    return bl;
 }
 
-// Block-wide argmin of (score, original index) over the live slots of [0, m0).  Every slot gets an FP32
-// estimate of its score first; only the slots within 1e-4 of the thread's best estimate are then scored
-// with the FP64 division, so the result (ties included) is the exact FP64 argmin.
+// Every thread holds at most one candidate (slot < 0: none).  Publishes the warp's best in the record buffer,
+// then, after the barrier, every warp derives the block's best from the records.
+template <int NT>
+__device__ __forceinline__ Pick block_pick(unsigned key, double s, int slot, int orig, double w, double dgv,
+                                           const Records& rec) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (slot < 0) key = KEY_NONE;
+    const int wl = warp_winner(key, s, orig);
+    if (wl < 0) { if (lane == 0) rec.key[warp] = KEY_NONE; }
+    else if (lane == wl) {
+        rec.key[warp] = key; rec.slot[warp] = slot; rec.orig[warp] = orig;
+        rec.s[warp] = s; rec.w[warp] = w; rec.dgv[warp] = dgv;
+    }
+    __syncthreads();
+    const bool in = lane < NW;
+    const unsigned k2 = in ? rec.key[lane] : KEY_NONE;
+    const double s2 = (in && k2 != KEY_NONE) ? rec.s[lane] : CUDART_INF;
+    const int o2 = (in && k2 != KEY_NONE) ? rec.orig[lane] : 0x7fffffff;
+    const int ww = warp_winner(k2, s2, o2);
+    Pick p;
+    p.slot = -1; p.orig = -1; p.w = 0.0; p.dgv = 0.0;
+    if (ww >= 0) { p.slot = rec.slot[ww]; p.orig = rec.orig[ww]; p.w = rec.w[ww]; p.dgv = rec.dgv[ww]; }
+    return p;
+}
+
+// The thread's best live slot among its own (slots tid, tid+NT, ...) by (score, original index).  Every slot
+// gets an FP32 estimate of its score first; only the slots within 1e-4 of the thread's best estimate are
+// scored with the FP64 division, so the result (ties included) is the exact FP64 choice.
+// With the outlier rule (Section 4, "Quantization Outliers") a slot whose error exceeds Delta/2 wins by
+// largest error; such candidates get keys below every regular one.
 template <int NT, int KMAX>
-__device__ void blk_argmin(const double* wd, const double* dg, const int* perm, int m0, bool quant, bool outliers,
-                           Bcast* bc, char* scratch) {
+__device__ __forceinline__ void thread_best(const double* wd, const double* dg, const int* perm, int m0, bool quant,
+                                            bool outliers, double sc, double ze, double mq,
+                                            unsigned* key, double* s_out, int* slot_out) {
     const int tid = threadIdx.x;
-    const double sc = bc->sc, ze = bc->ze, mq = bc->mq;
+    const double isc = 1.0 / sc;
     float sa[KMAX];
     float smin = CUDART_INF_F;
     double oe = -1.0;
@@ -101,7 +136,7 @@ __device__ void blk_argmin(const double* wd, const double* dg, const int* perm, 
         if (j < m0 && perm[j] >= 0) {
             const double w = wd[j];
             double err = -w, code;
-            if (quant) err = grid_q(w, sc, ze, mq, &code) - w;
+            if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
             sa[k] = __double2float_rn(err * err) / __double2float_rn(dg[j]);
             smin = fminf(smin, sa[k]);                       // fminf ignores a NaN estimate
             if (outliers) {
@@ -120,13 +155,18 @@ __device__ void blk_argmin(const double* wd, const double* dg, const int* perm, 
         if (sa[k] <= thr || (sa[k] == smin)) {               // false for NaN estimates and for idle lanes
             const double w = wd[j];
             double err = -w, code;
-            if (quant) err = grid_q(w, sc, ze, mq, &code) - w;
+            if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
             const double s = err * err / dg[j];
             const int o = perm[j];
             if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
         }
     }
-    blk_reduce_pick<NT>(bs, bo, bslot, oe, oo, oslot, outliers, bc, scratch);
+    *key = KEY_NONE; *s_out = bs; *slot_out = bslot;
+    if (bslot >= 0) *key = float_key(__double2float_rn(bs));
+    if (outliers && oslot >= 0) {
+        // an outlier precedes every regular candidate (scores are non-negative) and a larger error comes first
+        *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe));
+    }
 }
 
 // Applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts
@@ -224,6 +264,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     int* hl = reinterpret_cast<int*>(smem + BLK_OFF_HL);
     int* mv = reinterpret_cast<int*>(smem + BLK_OFF_MV);
     uint32_t* colmask = reinterpret_cast<uint32_t*>(smem + BLK_OFF_CM);
+    float* rf = reinterpret_cast<float*>(smem + BLK_OFF_RF);
     double* wd = reinterpret_cast<double*>(smem + BLK_FIXED);
     double* dg = wd + cap;
     int* perm = reinterpret_cast<int*>(dg + cap);
@@ -267,7 +308,6 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         }
         for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
         if (tid == 0) {
-            bc->fail = 0;
             bc->sc = 1.0; bc->ze = 0.0; bc->mq = 0.0;
             if (a.mode == MODE_QUANT) {
                 bc->sc = (double)a.scale[r]; bc->ze = (double)a.zero[r];
@@ -288,16 +328,19 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             }
         }
         __syncthreads();
+        double gsc = bc->sc, gze = bc->ze, gmq = bc->mq;       // grid parameters of the row (registers)
 
         int m0 = d;                      // slots in use (tail phase: number of live slots)
         int nb = 0;                      // pending vectors
         int ldz = (m0 + 7) & ~7;
         int bcur = min(a.max_pending, a.panel_floats / ldz);
         int s = 0;
+        bool failed = false;
         for (; s < total; ++s) {
             if (!tail) {
                 if (d > ms && nb > 0 && (nb == bcur || m0 - nb <= ms)) {
                     // ---- flush: apply the pending vectors and compact to m1 slots ------------------------
+                    __syncthreads();                           // the last step's vector and perm updates
                     const int m1 = m0 - nb;
                     if (tid == 0) {
                         int nh = 0, sp = m1;
@@ -357,121 +400,100 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
                     hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, off));
                 }
-                float* rf = reinterpret_cast<float*>(scratch);
                 if (lane == 0) { rf[warp] = lo; rf[32 + warp] = hi; }
                 __syncthreads();
-                if (tid == 0) {
-                    for (int k = 0; k < NW; ++k) { lo = fminf(lo, rf[k]); hi = fmaxf(hi, rf[32 + k]); }
-                    float sc, ze;
-                    grid_from_range(lo, hi, a.bits, a.symmetric, &sc, &ze);
-                    a.scale[r] = sc; a.zero[r] = ze;
-                    bc->sc = (double)sc; bc->ze = (double)ze; bc->mq = (double)grid_maxq(a.bits, a.symmetric);
-                }
-                __syncthreads();
+                for (int k = 0; k < NW; ++k) { lo = fminf(lo, rf[k]); hi = fmaxf(hi, rf[32 + k]); }
+                float sc, ze;
+                grid_from_range(lo, hi, a.bits, a.symmetric, &sc, &ze);
+                if (tid == 0) { a.scale[r] = sc; a.zero[r] = ze; }
+                gsc = (double)sc; gze = (double)ze; gmq = (double)grid_maxq(a.bits, a.symmetric);
+                __syncthreads();                               // rf is reused by the next row's grid
             }
-            // ---- pick the slot -------------------------------------------------------------------------
+            // ---- pick the slot: one candidate per thread, combined through the record buffer ------------
+            unsigned key = KEY_NONE;
+            double cs = 0.0;
+            int cslot = -1;
             if (forced) {
-                if (tid == 0) bc->slot = -1;
-                __syncthreads();
                 const int f = a.forced_order[(size_t)r * d + s];
                 for (int j = tid; j < m0; j += NT)
-                    if (perm[j] == f) bc->slot = j;
-                __syncthreads();
+                    if (perm[j] == f) { cslot = j; key = 0x80000000u; }
             } else {
-                blk_argmin<NT, KMAX>(wd, dg, perm, m0, q_now, outliers, bc, scratch);
+                thread_best<NT, KMAX>(wd, dg, perm, m0, q_now, outliers, gsc, gze, gmq, &key, &cs, &cslot);
             }
-            const int p = bc->slot;
-            if (tid == 0) {
-                int fail = 0;
-                double dpp = 0, e = 0, qp = 0, code = -1;
-                if (p < 0) fail = 1;
-                else {
-                    bc->op = perm[p];
-                    dpp = dg[p];
-                    if (!(dpp > 0.0) || !isfinite(dpp) || !isfinite(wd[p])) fail = 1;
-                    else {
-                        if (q_now) qp = grid_q(wd[p], bc->sc, bc->ze, bc->mq, &code);
-                        e = wd[p] - qp;
-                    }
-                }
-                bc->fail = fail; bc->dpp = dpp; bc->e = e; bc->qp = qp; bc->code = code;
-            }
+            const Records rec = rec_view(scratch, s & 1);
+            const Pick pk = block_pick<NT>(key, cs, cslot, cslot >= 0 ? perm[cslot] : -1,
+                                           cslot >= 0 ? wd[cslot] : 0.0, cslot >= 0 ? dg[cslot] : 0.0, rec);
+            const int p = pk.slot, op = pk.orig;
+            const double dpp = pk.dgv, wp = pk.w;
+            if (p < 0 || !(dpp > 0.0) || !isfinite(dpp) || !isfinite(wp)) { failed = true; break; }
+            double qp = 0.0, code = -1.0;
+            if (q_now) qp = grid_q(wp, gsc, gze, gmq, &code);
+            const double e = wp - qp;
             if (!tail) {
                 // ======================= deferred-update step ==============================================
                 float* zb = panel + (size_t)nb * ldz;
-                if (p >= 0) {
-                    // pivot column of the stored matrix, corrected by the pending vectors
-                    float c[KMAX], corr[KMAX];
-                    const float* rowp = Hp + (size_t)p * ldp;
+                // pivot column of the stored matrix (own slots), corrected by the pending vectors
+                float c[KMAX], corr[KMAX];
+                const float* rowp = Hp + (size_t)p * ldp;
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) {
+                    const int j = tid + k * NT;
+                    c[k] = 0.f; corr[k] = 0.f;
+                    if (j < m0 && perm[j] >= 0) c[k] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                }
+                const double idpp = 1.0 / dpp;
+                const double f = e * idpp;
+                const float rs = __frsqrt_rn((float)dpp);
+                for (int b = 0; b < nb; ++b) {
+                    const float* zo = panel + (size_t)b * ldz;
+                    const float zp = zo[p];
 #pragma unroll
                     for (int k = 0; k < KMAX; ++k) {
                         const int j = tid + k * NT;
-                        c[k] = 0.f; corr[k] = 0.f;
-                        if (j < m0 && perm[j] >= 0) c[k] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
-                    }
-                    for (int b = 0; b < nb; ++b) {
-                        const float* zo = panel + (size_t)b * ldz;
-                        const float zp = zo[p];
-#pragma unroll
-                        for (int k = 0; k < KMAX; ++k) {
-                            const int j = tid + k * NT;
-                            if (j < m0) corr[k] = fmaf(zo[j], zp, corr[k]);
-                        }
-                    }
-#pragma unroll
-                    for (int k = 0; k < KMAX; ++k) {
-                        const int j = tid + k * NT;
-                        if (j < m0) zb[j] = (perm[j] >= 0) ? c[k] - corr[k] : 0.f;
+                        if (j < m0) corr[k] = fmaf(zo[j], zp, corr[k]);
                     }
                 }
-                __syncthreads();
-                if (bc->fail) break;
-                {
-                    const double dpp = bc->dpp, f = bc->e / dpp, idpp = 1.0 / dpp;
-                    const float rs = (float)(1.0 / sqrt(dpp));
-                    const int op = bc->op;
 #pragma unroll
-                    for (int k = 0; k < KMAX; ++k) {
-                        const int j = tid + k * NT;
-                        if (j >= m0 || perm[j] < 0) continue;
-                        if (j == p) { zb[j] = 0.f; perm[j] = -1; continue; }
-                        const float vj = zb[j];
-                        const double nw = wd[j] - f * (double)vj;
-                        wd[j] = nw;
-                        dg[j] -= (double)vj * (double)vj * idpp;
-                        zb[j] = vj * rs;
-                        if (has_wfull) wfull[perm[j]] = (float)nw;
+                for (int k = 0; k < KMAX; ++k) {
+                    const int j = tid + k * NT;
+                    if (j >= m0) continue;
+                    if (perm[j] < 0) { zb[j] = 0.f; continue; }
+                    if (j == p) { zb[j] = 0.f; perm[j] = -1; continue; }
+                    const float vj = c[k] - corr[k];
+                    const double nw = wd[j] - f * (double)vj;
+                    wd[j] = nw;
+                    dg[j] -= (double)vj * (double)vj * idpp;
+                    zb[j] = vj * rs;
+                    if (has_wfull) wfull[perm[j]] = (float)nw;
+                }
+                if (tid == 0) {
+                    pv[nb] = p;
+                    if (has_wfull) wfull[op] = (float)qp;
+                    if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)qp;
+                    if (!forced) {
+                        const int t = s - n_forced;
+                        if (a.order) a.order[(size_t)r * d + t] = op;
+                        if (a.loss) a.loss[(size_t)r * d + t] = (float)(e * e / dpp);
                     }
-                    if (tid == 0) {
-                        pv[nb] = p;
-                        if (has_wfull) wfull[op] = (float)bc->qp;
-                        if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)bc->qp;
-                        if (!forced) {
-                            const int t = s - n_forced;
-                            if (a.order) a.order[(size_t)r * d + t] = op;
-                            if (a.loss) a.loss[(size_t)r * d + t] = (float)(bc->e * bc->e / dpp);
-                        }
-                        if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)bc->code;
-                    }
+                    if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)code;
                 }
                 ++nb;
-                __syncthreads();
-                if (a.w_trace && s < a.trace_steps)
+                if (a.w_trace && s < a.trace_steps) {
+                    __syncthreads();
                     for (int j = tid; j < d; j += NT)
                         a.w_trace[((size_t)r * (a.trace_steps + 1) + s + 1) * d + j] = wfull[j];
+                    __syncthreads();                           // wfull is written again in the next step
+                }
             } else {
                 // ======================= on-chip step (compaction at every step) ===========================
                 const int m = m0, last = m0 - 1;
-                if (p >= 0)
-                    for (int j = tid; j < m; j += NT) {
-                        tv[j] = (j <= p) ? S[p * lds + j] : S[j * lds + p];
-                        tlr[j] = S[last * lds + j];
-                    }
+                for (int j = tid; j < m; j += NT) {
+                    tv[j] = (j <= p) ? S[p * lds + j] : S[j * lds + p];
+                    tlr[j] = S[last * lds + j];
+                }
                 __syncthreads();
-                if (bc->fail) break;
                 {
-                    const double dpp = bc->dpp, f = bc->e / dpp;
-                    const int op = bc->op;
+                    const double f = e / dpp;
                     for (int j = tid; j < m; j += NT) {
                         if (j == p) continue;
                         const float vj = tv[j];
@@ -485,14 +507,14 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         if (j == last) { perm[p] = oj; tv[p] = vj; tlr[p] = tlr[last]; }
                     }
                     if (tid == 0) {
-                        if (has_wfull) wfull[op] = (float)bc->qp;
-                        if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)bc->qp;
+                        if (has_wfull) wfull[op] = (float)qp;
+                        if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)qp;
                         if (!forced) {
                             const int t = s - n_forced;
                             if (a.order) a.order[(size_t)r * d + t] = op;
-                            if (a.loss) a.loss[(size_t)r * d + t] = (float)(bc->e * bc->e / dpp);
+                            if (a.loss) a.loss[(size_t)r * d + t] = (float)(e * e / dpp);
                         }
-                        if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)bc->code;
+                        if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)code;
                     }
                 }
                 __syncthreads();
@@ -506,7 +528,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             }
         }
         // ---- row epilogue ---------------------------------------------------------------------------------
-        if (s < total) {        // stopped early: report the step, mark what was not produced
+        __syncthreads();
+        if (failed) {           // stopped early: report the step, mark what was not produced
             if (tid == 0) a.row_status[r] = 1 + s;
             const int t0 = (s < n_forced) ? 0 : s - n_forced;
             for (int t = t0 + tid; t < n_free; t += NT) {
@@ -575,6 +598,18 @@ size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di
     int blocks = di.sm_count * 4;                 // the largest grid any thread-count choice uses
     if (row_count > 0 && row_count < blocks) blocks = row_count;
     return round_up((size_t)blocks * d * cap * sizeof(float), 256);
+}
+
+obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
+    DeviceInfo di;
+    obc_status st = device_info(&di);
+    if (st != OBC_OK) return st;
+    BlkPlan p;
+    if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p)) return OBC_ERR_UNSUPPORTED;
+    const int mp = engine_pending_choice();
+    plan[0] = OBC_ENGINE_BLOCKED; plan[1] = p.nt; plan[2] = p.per_sm; plan[3] = p.ms; plan[4] = p.panel_floats;
+    plan[5] = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB; plan[6] = di.sm_count; plan[7] = 0;
+    return OBC_OK;
 }
 
 template <int NT, int KMAX>
