@@ -89,7 +89,7 @@ obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
  * plan (host int32[8]): [0] engine (OBC_ENGINE_STREAMING or OBC_ENGINE_BLOCKED), [1] threads per row,
  * [2] rows resident per SM, [3] active size at which a row moves into shared memory, [4] floats of shared memory
  * for deferred update vectors (BLOCKED), [5] limit on deferred updates (BLOCKED), [6] SM count, [7] 0.
- * A BLOCKED row of current size m defers min(plan[5], plan[4] / round_up(m, 8)) updates between two passes over
+ * A BLOCKED row of current size m defers min(plan[5], plan[4] / round_up(m, 16)) updates between two passes over
  * its matrix.  Used by the benchmark to state the bytes a launch has to move. */
 obc_status obc_engine_plan(int d_col, int with_trace, int32_t *plan);
 

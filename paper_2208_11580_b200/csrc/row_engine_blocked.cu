@@ -15,13 +15,14 @@
 // vectors and compacts at the same time: a dead slot h below the new size m1 is taken over by a live slot
 // s >= m1, i.e. element (i, j) of the new triangle is read from (max(si, sj), min(si, sj)) of the old one.
 // All such foreign reads come from rows >= m1, which the flush never writes, so it runs in place.
-// The flush works on warp tiles of 8 rows x 128 columns with the 8 x 4 sub-tile of each lane in registers;
+// The flush works on warp tiles of 16 rows x 128 columns with the 16 x 4 sub-tile of each lane in registers;
 // the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
 // the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
 // finishes on chip with step-by-step updates.
 //
-// Step protocol.  Between two flushes slot j belongs to thread j mod NT, which is the only one to touch
-// wd[j], dg[j], perm[j] and its entries of the pending vectors.  Each thread proposes its best slot, the
+// Step protocol.  Between two flushes every slot belongs to one thread (groups of 4 consecutive slots per
+// thread), which is the only one to touch wd[j], dg[j], perm[j] and its entries of the pending vectors; the
+// update phase also leaves an FP32 estimate of each own slot's next score in registers.  Each thread proposes its best slot, the
 // warps combine the proposals and publish one record per warp (with the candidate's weight and diagonal),
 // and after the single barrier of the step every warp reads the records and derives the same winner, so
 // no second barrier is needed to announce it.  Records alternate between two buffers by step parity.
@@ -114,82 +115,95 @@ __device__ __forceinline__ Pick block_pick(unsigned key, double s, int slot, int
     return p;
 }
 
-// The thread's best live slot among its own (slots tid, tid+NT, ...) by (score, original index).  Every slot
-// gets an FP32 estimate of its score first; only the slots within 1e-4 of the thread's best estimate are
-// scored with the FP64 division, so the result (ties included) is the exact FP64 choice.
-// With the outlier rule (Section 4, "Quantization Outliers") a slot whose error exceeds Delta/2 wins by
-// largest error; such candidates get keys below every regular one.
+// Slot ownership between two flushes: thread t owns the slots 4t .. 4t+3 of every group of 4 NT slots, i.e.
+// slot(k) = (k / 4) * 4 NT + 4 t + (k % 4) for k < KMAX, so that its entries of a pending vector, of a matrix
+// row and of the state arrays are 16 contiguous bytes.
+template <int NT>
+__device__ __forceinline__ int own_slot(int k) { return (k >> 2) * (4 * NT) + (threadIdx.x << 2) + (k & 3); }
+
+// FP32 estimate of the score of a slot (relative error of a few 1e-7): it only screens candidates, the slots
+// within 1e-4 of the thread's best estimate are scored again with the FP64 division.
+__device__ __forceinline__ float score_estimate(double w, double dgv, bool quant, double sc, double isc, double ze,
+                                                double mq) {
+    double err = -w, code;
+    if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
+    return __fdividef(__double2float_rn(err * err), __double2float_rn(dgv));
+}
+
+// Estimates of all own slots from the state arrays (NaN for dead or unused slots).
 template <int NT, int KMAX>
-__device__ __forceinline__ void thread_best(const double* wd, const double* dg, const int* perm, int m0, bool quant,
-                                            bool outliers, double sc, double ze, double mq,
-                                            unsigned* key, double* s_out, int* slot_out) {
-    const int tid = threadIdx.x;
-    const double isc = 1.0 / sc;
-    float sa[KMAX];
-    float smin = CUDART_INF_F;
-    double oe = -1.0;
-    int oo = 0x7fffffff, oslot = -1;
+__device__ __forceinline__ void estimate_own(float (&sa)[KMAX], const double* wd, const double* dg, const int* perm,
+                                             int m0, bool quant, double sc, double isc, double ze, double mq) {
 #pragma unroll
     for (int k = 0; k < KMAX; ++k) {
-        const int j = tid + k * NT;
+        const int j = own_slot<NT>(k);
         sa[k] = CUDART_NAN_F;
-        if (j < m0 && perm[j] >= 0) {
+        if (j < m0 && perm[j] >= 0) sa[k] = score_estimate(wd[j], dg[j], quant, sc, isc, ze, mq);
+    }
+}
+
+// The thread's best live slot among its own by (score, original index), given the estimates: only the slots
+// within 1e-4 of the thread's best estimate take the FP64 division, so the result (ties included) is the
+// exact FP64 choice.  With the outlier rule (Section 4, "Quantization Outliers") a slot whose error exceeds
+// Delta/2 wins by largest error; such candidates get negative scores, below every regular one.
+template <int NT, int KMAX>
+__device__ __forceinline__ void thread_best(const float (&sa)[KMAX], const double* wd, const double* dg,
+                                            const int* perm, bool quant, bool outliers, double sc, double isc,
+                                            double ze, double mq, unsigned* key, double* s_out, int* slot_out) {
+    float smin = CUDART_INF_F;
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) smin = fminf(smin, sa[k]);           // fminf ignores NaN estimates
+    const float thr = smin + 1e-4f * fabsf(smin);
+    double bs = CUDART_INF, oe = -1.0;
+    int bo = 0x7fffffff, bslot = -1, oo = 0x7fffffff, oslot = -1;
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+        const bool cand = sa[k] <= thr || sa[k] == smin;                 // false for NaN estimates
+        if (cand || (outliers && sa[k] == sa[k])) {
+            const int j = own_slot<NT>(k);
             const double w = wd[j];
             double err = -w, code;
             if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
-            sa[k] = __double2float_rn(err * err) / __double2float_rn(dg[j]);
-            smin = fminf(smin, sa[k]);                       // fminf ignores a NaN estimate
+            const int o = perm[j];
+            if (cand) {
+                const double s = err * err / dg[j];
+                if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
+            }
             if (outliers) {
                 const double a = fabs(err);
-                const int o = perm[j];
                 if (a > 0.5 * sc && (a > oe || (a == oe && o < oo))) { oe = a; oo = o; oslot = j; }
             }
         }
     }
-    const float thr = smin + 1e-4f * fabsf(smin);
-    double bs = CUDART_INF;
-    int bo = 0x7fffffff, bslot = -1;
-#pragma unroll
-    for (int k = 0; k < KMAX; ++k) {
-        const int j = tid + k * NT;
-        if (sa[k] <= thr || (sa[k] == smin)) {               // false for NaN estimates and for idle lanes
-            const double w = wd[j];
-            double err = -w, code;
-            if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
-            const double s = err * err / dg[j];
-            const int o = perm[j];
-            if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
-        }
-    }
     *key = KEY_NONE; *s_out = bs; *slot_out = bslot;
     if (bslot >= 0) *key = float_key(__double2float_rn(bs));
-    if (outliers && oslot >= 0) {
-        // an outlier precedes every regular candidate (scores are non-negative) and a larger error comes first
-        *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe));
-    }
+    if (outliers && oslot >= 0) { *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe)); }
 }
 
 // Applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts
 // it to m1 rows.  srcm[i] = old slot whose data new slot i takes (i itself unless i is a hole).
-template <int NT>
+// A warp works on tiles of RG rows x 128 columns (row groups dealt out cyclically to the warps); each lane keeps
+// its RG x 4 sub-tile in registers, so RG x 16 bytes per lane are in flight while a tile is fetched and the
+// pending vectors cost RG/4 + 1 shared-memory loads per 4 RG multiply-adds.
+template <int NT, int RG>
 __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m1, int nb, const float* Z, int ldz,
                                           const unsigned short* srcm, const uint32_t* colmask) {
     constexpr int NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nrg = (m1 + 7) >> 3;
+    const int nrg = (m1 + RG - 1) / RG;
     for (int rg = warp; rg < nrg; rg += NW) {
-        const int i0 = rg << 3;
-        const int nrows = min(8, m1 - i0);
-        int sr[8];
+        const int i0 = rg * RG;
+        const int nrows = min(RG, m1 - i0);
+        int sr[RG];
 #pragma unroll
-        for (int r = 0; r < 8; ++r) sr[r] = (r < nrows) ? (int)srcm[i0 + r] : i0;
+        for (int r = 0; r < RG; ++r) sr[r] = (r < nrows) ? (int)srcm[i0 + r] : i0;
         const int jend = i0 + nrows;                           // columns [0, jend) hold data of this row group
         for (int c0 = 0; c0 < jend; c0 += 128) {
             const int j = c0 + (lane << 2);
             if (j >= jend) continue;                           // whole float4 above the diagonal of every row
-            float4 acc[8];
+            float4 acc[RG];
 #pragma unroll
-            for (int r = 0; r < 8; ++r) {
+            for (int r = 0; r < RG; ++r) {
                 acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (r < nrows && j <= i0 + r)
                     acc[r] = *reinterpret_cast<const float4*>(Hp + (size_t)sr[r] * ldp + j);
@@ -203,7 +217,7 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
                     const int jj = j + comp;
                     const int sj = (int)srcm[jj];
 #pragma unroll
-                    for (int r = 0; r < 8; ++r) {
+                    for (int r = 0; r < RG; ++r) {
                         if (r < nrows && jj <= i0 + r) {
                             const int hi = max(sr[r], sj), lo = min(sr[r], sj);
                             const float val = Hp[(size_t)hi * ldp + lo];
@@ -215,20 +229,23 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
             }
             for (int b = 0; b < nb; ++b) {
                 const float* zb = Z + (size_t)b * ldz;
-                const float4 za = *reinterpret_cast<const float4*>(zb + i0);
-                const float4 zc = *reinterpret_cast<const float4*>(zb + i0 + 4);
                 const float4 zj = *reinterpret_cast<const float4*>(zb + j);
-                const float zi[8] = {za.x, za.y, za.z, za.w, zc.x, zc.y, zc.z, zc.w};
 #pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    acc[r].x = fmaf(-zi[r], zj.x, acc[r].x);
-                    acc[r].y = fmaf(-zi[r], zj.y, acc[r].y);
-                    acc[r].z = fmaf(-zi[r], zj.z, acc[r].z);
-                    acc[r].w = fmaf(-zi[r], zj.w, acc[r].w);
+                for (int r4 = 0; r4 < RG / 4; ++r4) {
+                    const float4 za = *reinterpret_cast<const float4*>(zb + i0 + 4 * r4);
+                    const float zi[4] = {za.x, za.y, za.z, za.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float4& t = acc[4 * r4 + q];
+                        t.x = fmaf(-zi[q], zj.x, t.x);
+                        t.y = fmaf(-zi[q], zj.y, t.y);
+                        t.z = fmaf(-zi[q], zj.z, t.z);
+                        t.w = fmaf(-zi[q], zj.w, t.w);
+                    }
                 }
             }
 #pragma unroll
-            for (int r = 0; r < 8; ++r)
+            for (int r = 0; r < RG; ++r)
                 if (r < nrows && j <= i0 + r)
                     *reinterpret_cast<float4*>(Hp + (size_t)(i0 + r) * ldp + j) = acc[r];
         }
@@ -306,6 +323,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             if (has_wfull) wfull[j] = w;
             if (a.codes) a.codes[(size_t)r * d + j] = -1;
         }
+        for (int j = d + tid; j < cap; j += NT) perm[j] = -1;
         for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
         if (tid == 0) {
             bc->sc = 1.0; bc->ze = 0.0; bc->mq = 0.0;
@@ -332,10 +350,13 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 
         int m0 = d;                      // slots in use (tail phase: number of live slots)
         int nb = 0;                      // pending vectors
-        int ldz = (m0 + 7) & ~7;
+        int ldz = (m0 + 15) & ~15;
         int bcur = min(a.max_pending, a.panel_floats / ldz);
         int s = 0;
         bool failed = false;
+        float sa[KMAX];                  // score estimates of the own slots, kept up to date by the update phase
+        bool sa_valid = false;
+        double gisc = 1.0 / gsc;
         for (; s < total; ++s) {
             if (!tail) {
                 if (d > ms && nb > 0 && (nb == bcur || m0 - nb <= ms)) {
@@ -365,7 +386,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         atomicOr(&colmask[h >> 5], 1u << (h & 31));
                     }
                     __syncthreads();
-                    blk_flush<NT>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
+                    blk_flush<NT, 16>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
                     __syncthreads();
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
@@ -374,7 +395,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         colmask[h >> 5] = 0u;
                     }
                     m0 = m1; nb = 0;
-                    ldz = (m0 + 7) & ~7;
+                    sa_valid = false;
+#pragma unroll
+                    for (int k = 0; k < KMAX; ++k) sa[k] = CUDART_NAN_F;      // slots changed hands: not carried over
+                    ldz = (m0 + 15) & ~15;
                     bcur = min(a.max_pending, a.panel_floats / ldz);
                     __syncthreads();
                 }
@@ -393,8 +417,11 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             // ---- grid of the compound path: built from the survivors when the replay is over -----------
             if (a.mode == MODE_REPLAY_QUANT && s == n_forced) {
                 float lo = 0.f, hi = 0.f;
-                for (int j = tid; j < m0; j += NT)
-                    if (perm[j] >= 0) { const float w = (float)wd[j]; lo = fminf(lo, w); hi = fmaxf(hi, w); }
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) {               // own slots: their owner is the only writer
+                    const int j = own_slot<NT>(k);
+                    if (j < m0 && perm[j] >= 0) { const float w = (float)wd[j]; lo = fminf(lo, w); hi = fmaxf(hi, w); }
+                }
 #pragma unroll
                 for (int off = 16; off; off >>= 1) {
                     lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, off));
@@ -407,6 +434,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 grid_from_range(lo, hi, a.bits, a.symmetric, &sc, &ze);
                 if (tid == 0) { a.scale[r] = sc; a.zero[r] = ze; }
                 gsc = (double)sc; gze = (double)ze; gmq = (double)grid_maxq(a.bits, a.symmetric);
+                gisc = 1.0 / gsc;
+                sa_valid = false;
                 __syncthreads();                               // rf is reused by the next row's grid
             }
             // ---- pick the slot: one candidate per thread, combined through the record buffer ------------
@@ -415,10 +444,15 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             int cslot = -1;
             if (forced) {
                 const int f = a.forced_order[(size_t)r * d + s];
-                for (int j = tid; j < m0; j += NT)
-                    if (perm[j] == f) { cslot = j; key = 0x80000000u; }
+#pragma unroll
+                for (int k = 0; k < KMAX; ++k) {
+                    const int j = own_slot<NT>(k);
+                    if (j < m0 && perm[j] == f) { cslot = j; key = 0x80000000u; }
+                }
             } else {
-                thread_best<NT, KMAX>(wd, dg, perm, m0, q_now, outliers, gsc, gze, gmq, &key, &cs, &cslot);
+                if (!sa_valid || tail || outliers)
+                    estimate_own<NT, KMAX>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq);
+                thread_best<NT, KMAX>(sa, wd, dg, perm, q_now, outliers, gsc, gisc, gze, gmq, &key, &cs, &cslot);
             }
             const Records rec = rec_view(scratch, s & 1);
             const Pick pk = block_pick<NT>(key, cs, cslot, cslot >= 0 ? perm[cslot] : -1,
@@ -434,12 +468,29 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 float* zb = panel + (size_t)nb * ldz;
                 // pivot column of the stored matrix (own slots), corrected by the pending vectors
                 float c[KMAX], corr[KMAX];
+                unsigned live = 0u;
                 const float* rowp = Hp + (size_t)p * ldp;
 #pragma unroll
-                for (int k = 0; k < KMAX; ++k) {
-                    const int j = tid + k * NT;
-                    c[k] = 0.f; corr[k] = 0.f;
-                    if (j < m0 && perm[j] >= 0) c[k] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                for (int g = 0; g < KMAX / 4; ++g) {
+                    const int jb = own_slot<NT>(4 * g);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) { c[4 * g + q] = 0.f; corr[4 * g + q] = 0.f; }
+                    if (jb >= m0) continue;
+                    const int4 pm = *reinterpret_cast<const int4*>(perm + jb);
+                    const int pq[4] = {pm.x, pm.y, pm.z, pm.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (jb + q < m0 && pq[q] >= 0) live |= 1u << (4 * g + q);
+                    if (jb + 3 <= p) {
+                        const float4 v = *reinterpret_cast<const float4*>(rowp + jb);
+                        c[4 * g] = v.x; c[4 * g + 1] = v.y; c[4 * g + 2] = v.z; c[4 * g + 3] = v.w;
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int j = jb + q;
+                            if ((live >> (4 * g + q)) & 1u) c[4 * g + q] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                        }
+                    }
                 }
                 const double idpp = 1.0 / dpp;
                 const double f = e * idpp;
@@ -448,24 +499,43 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     const float* zo = panel + (size_t)b * ldz;
                     const float zp = zo[p];
 #pragma unroll
-                    for (int k = 0; k < KMAX; ++k) {
-                        const int j = tid + k * NT;
-                        if (j < m0) corr[k] = fmaf(zo[j], zp, corr[k]);
+                    for (int g = 0; g < KMAX / 4; ++g) {
+                        if ((live >> (4 * g)) & 0xFu) {
+                            const float4 z = *reinterpret_cast<const float4*>(zo + own_slot<NT>(4 * g));
+                            corr[4 * g] = fmaf(z.x, zp, corr[4 * g]);
+                            corr[4 * g + 1] = fmaf(z.y, zp, corr[4 * g + 1]);
+                            corr[4 * g + 2] = fmaf(z.z, zp, corr[4 * g + 2]);
+                            corr[4 * g + 3] = fmaf(z.w, zp, corr[4 * g + 3]);
+                        }
                     }
                 }
+                // state update of the own slots (Eq. 3 / Eq. 7), the new pending vector, and the score
+                // estimates the next free step starts from
+                const bool est_next = (s + 1 >= n_forced) && !outliers;
+                const bool q_next = quant && (s + 1 >= n_forced);
 #pragma unroll
-                for (int k = 0; k < KMAX; ++k) {
-                    const int j = tid + k * NT;
-                    if (j >= m0) continue;
-                    if (perm[j] < 0) { zb[j] = 0.f; continue; }
-                    if (j == p) { zb[j] = 0.f; perm[j] = -1; continue; }
-                    const float vj = c[k] - corr[k];
-                    const double nw = wd[j] - f * (double)vj;
-                    wd[j] = nw;
-                    dg[j] -= (double)vj * (double)vj * idpp;
-                    zb[j] = vj * rs;
-                    if (has_wfull) wfull[perm[j]] = (float)nw;
+                for (int g = 0; g < KMAX / 4; ++g) {
+                    const int jb = own_slot<NT>(4 * g);
+                    if (jb >= m0) continue;
+                    float zv[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int k = 4 * g + q, j = jb + q;
+                        zv[q] = 0.f;
+                        sa[k] = CUDART_NAN_F;
+                        if (!((live >> k) & 1u)) continue;
+                        if (j == p) { perm[j] = -1; continue; }
+                        const float vj = c[k] - corr[k];
+                        const double nw = wd[j] - f * (double)vj;
+                        const double nd = dg[j] - (double)vj * (double)vj * idpp;
+                        wd[j] = nw; dg[j] = nd;
+                        zv[q] = vj * rs;
+                        if (est_next) sa[k] = score_estimate(nw, nd, q_next, gsc, gisc, gze, gmq);
+                        if (has_wfull) wfull[perm[j]] = (float)nw;
+                    }
+                    *reinterpret_cast<float4*>(zb + jb) = make_float4(zv[0], zv[1], zv[2], zv[3]);
                 }
+                sa_valid = est_next;
                 if (tid == 0) {
                     pv[nb] = p;
                     if (has_wfull) wfull[op] = (float)qp;
@@ -576,7 +646,7 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out) {
     size_t share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
     if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
     const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull);
-    const size_t min_panel = (size_t)4 * ((cap + 7) & ~7);
+    const size_t min_panel = (size_t)4 * ((cap + 15) & ~15);
     while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
         p.per_sm >>= 1;
         share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
@@ -645,7 +715,7 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     }
     if (p.nt == 128) return blk_launch<128, 8>(a, blocks, p.smem, stream);
     if (p.nt == 256) return blk_launch<256, 8>(a, blocks, p.smem, stream);
-    return blk_launch<512, 10>(a, blocks, p.smem, stream);
+    return blk_launch<512, 12>(a, blocks, p.smem, stream);
 }
 
 }  // namespace obc
