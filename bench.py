@@ -34,9 +34,12 @@ METRIC = "eliminated_weights_per_s"
 UNIT = "weights/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per algorithmic byte of the row engine, from the ncu capture summarised in
-# profiles/row_engine_d1152_rows148_ncu_full.txt (287.8 GB moved for 603.3 GB of 8 m^2 model bytes); the
+# profiles/streaming_engine_d1152_rows148_ncu_full.txt (287.8 GB moved for 603.3 GB of 8 m^2 model bytes); the
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 287.8 / 603.3
+# The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 118.9 GB moved for 96.8 GB.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 118.9 / 96.8
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
@@ -362,8 +365,9 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
                 "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
-                "traffic": (None if blocked else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE)),
-                "traffic_source": ("see profiles/ for the ncu DRAM counters of this kernel on a smaller case" if blocked else
+                "traffic": int(own_bytes / n_eng * BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE) if blocked
+                           else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
+                "traffic_source": ("scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes" if blocked else
                                    "scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
                 "algorithmic_bytes_per_launch": int(own_bytes // n_eng), "ms_per_launch": round(eng_ms / n_eng, 3),
                 "launches_timed": len(engine_runs),
