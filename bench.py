@@ -145,13 +145,17 @@ class ClockSampler:
 class Layer:
     """Device buffers and the stage sequence of one workload, all through the C ABI."""
 
-    def __init__(self, name: str, W: np.ndarray, X: np.ndarray, dev, prec: int):
+    def __init__(self, name: str, W: np.ndarray, X: np.ndarray, dev, prec: int, row_begin: int = 0, row_count: int | None = None,
+                 group_world: int = 1):
         import torch
         import paper_2208_11580_b200 as obc
         self.obc, self.torch, self.name, self.dev, self.prec = obc, torch, name, dev, prec
         self.spec = obc_synth.SPECS[name]
         self.R, self.d = W.shape
         self.n = X.shape[1]
+        # rows this process eliminates (all of them unless one layer is sharded over several GPUs)
+        self.rb, self.rc = row_begin, (W.shape[0] - row_begin if row_count is None else row_count)
+        self.group_world = group_world
         R, d = self.R, self.d
         t = torch
         self.W = t.empty(R, d, dtype=t.float32, device=dev)
@@ -177,14 +181,14 @@ class Layer:
             self.Wq = t.zeros(R, d, dtype=t.float32, device=dev)
             self.codes = t.zeros(R, d, dtype=t.int32, device=dev)
         need = max(obc.obc_workspace_bytes(obc.OP_HESSIAN, 0, d, self.n), obc.obc_workspace_bytes(obc.OP_INVERSE, 0, d),
-                   obc.obc_workspace_bytes(obc.OP_PRUNE_TRACE, R, d), obc.obc_workspace_bytes(obc.OP_SELECT, R, d))
+                   obc.obc_workspace_bytes(obc.OP_PRUNE_TRACE, max(1, self.rc), d), obc.obc_workspace_bytes(obc.OP_SELECT, R, d))
         self.ws = t.empty(need, dtype=t.uint8, device=dev)
         self.W.copy_(t.from_numpy(W))
         self.X.copy_(t.from_numpy(X))
         self.engine_ms = []          # (label, CUDA-event ms, launch info) per engine launch since reset_timers()
         self._info = {}
         self._pending = []
-        self.eliminated = R * d * (2 if task == "prune+quant" else 1)
+        self.eliminated = self.rc * d * (2 if task == "prune+quant" else 1)
 
     def _timed(self, label, nbytes, fn):
         t = self.torch
@@ -203,25 +207,33 @@ class Layer:
         if task in ("prune", "prune+quant", "compound"):
             full_t = self.launch_info(with_trace=self.trace is not None)
             self._timed("engine:prune_trace", full_t, lambda: o.obc_prune_trace(self.W, self.Hinv, self.order, self.loss, self.status,
-                                                                              w_trace=self.trace, ws=self.ws))
+                                                                              w_trace=self.trace, row_begin=self.rb, row_count=self.rc, ws=self.ws))
+            if self.group_world > 1:   # the one exchange step of a row-sharded layer: traces of all rows to every rank
+                self._timed("exchange", 0, self._exchange)
             for i, k in enumerate(self.ks):
                 self._timed("select", 0, lambda i=i, k=k: o.obc_select_global_mask(self.loss, self.order, k, self.counts[i], self.masks[i], ws=self.ws))
                 if task != "compound":
                     self._timed("apply", 0, lambda i=i: o.obc_prune_apply(self.W, self.Hinv, self.order, self.counts[i], self.What[i], self.status,
-                                                                           w_trace=self.trace, trace_steps=d, ws=self.ws))
+                                                                           w_trace=self.trace, trace_steps=d, row_begin=self.rb, row_count=self.rc, ws=self.ws))
         if task in ("quant", "prune+quant"):
             self._timed("grid", 0, lambda: o.obc_minmax_grid(self.W, self.spec.bits, self.spec.symmetric, self.scale, self.zero))
             self._timed("engine:quantize", full, lambda: o.obc_quantize(self.W, self.Hinv, self.scale, self.zero, self.spec.bits, self.spec.symmetric,
-                                                                        self.Wq, self.codes, self.status, ws=self.ws))
+                                                                        self.Wq, self.codes, self.status, row_begin=self.rb, row_count=self.rc, ws=self.ws))
         if task == "compound":
             # replay of counts[r] pruning steps + quantisation of the survivors: again every size d..1 once per row
             self._timed("engine:replay_quantize", full, lambda: o.obc_quantize(
                 self.W, self.Hinv, self.scale, self.zero, self.spec.bits, self.spec.symmetric, self.Wq, self.codes, self.status,
-                prune_order=self.order, prune_counts=self.counts[0], ws=self.ws))
+                prune_order=self.order, prune_counts=self.counts[0], row_begin=self.rb, row_count=self.rc, ws=self.ws))
+
+    def _exchange(self):
+        from paper_2208_11580_b200.sharding import gather_traces
+        L, P = gather_traces(self.loss[self.rb:self.rb + self.rc], self.order[self.rb:self.rb + self.rc], self.R)
+        self.loss.copy_(L)
+        self.order.copy_(P)
 
     def launch_info(self, with_trace: bool):
         """What one engine launch over all rows (every active size d..1 once per row) has to move and compute."""
-        R, d = self.R, self.d
+        R, d = self.rc, self.d
         key = bool(with_trace)
         if key not in self._info:
             plan = self.obc.obc_engine_plan(d, with_trace)
@@ -282,7 +294,12 @@ def run_ours(args):
     name = args.workload
     W, X, spec = obc_synth.make_layer(name)          # every rank compresses its own copy of the layer
     prec = {"fp32": obc.PREC_FP32, "tf32": obc.PREC_TF32, "bf16x3": obc.PREC_BF16X3}[args.hessian_prec]
-    layer = Layer(name, W, X, dev, prec)
+    if args.shard_rows and world > 1:
+        from paper_2208_11580_b200.sharding import row_range
+        rb, rc = row_range(W.shape[0], world, rank)        # ONE layer, its rows split over the GPUs
+        layer = Layer(name, W, X, dev, prec, rb, rc, world)
+    else:
+        layer = Layer(name, W, X, dev, prec)                 # every GPU compresses its own copy of the layer
 
     def barrier():
         if world > 1:
@@ -316,7 +333,9 @@ def run_ours(args):
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         total_ms = float(tmax.item())
     ms_per_step = total_ms / args.steps
-    value = world * layer.eliminated / (ms_per_step * 1e-3)
+    sharded = args.shard_rows and world > 1
+    total_units = layer.R * layer.d * (2 if spec.task == "prune+quant" else 1) * (1 if sharded else world)
+    value = total_units / (ms_per_step * 1e-3)
 
     # ---- end to end: pinned host inputs -> device, hot path, results -> pinned host, every step ---------------------
     t = torch
@@ -345,7 +364,7 @@ def run_ours(args):
         tmax = torch.tensor([e2e_ms], device=dev)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         e2e_ms = float(tmax.item())
-    e2e_value = world * layer.eliminated / (e2e_ms / e2e_steps * 1e-3)
+    e2e_value = total_units / (e2e_ms / e2e_steps * 1e-3)
 
     if rank != 0:
         if world > 1:
@@ -387,14 +406,15 @@ def run_ours(args):
         roofline["streaming_engine"] = streaming_reference(layer, peak)
     cpu = cpu_baseline(name, W, layer.Hinv.cpu().numpy(), layer, args.cpu_seconds)
     out = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-           "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
-           "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True,
+           "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
            "config": {"workload": f"{name}: {spec.note}", "d_row": layer.R, "d_col": layer.d, "n_calib": layer.n,
                       "task": spec.task, "bits": spec.bits, "sparsities": list(spec.sparsities),
                       "hessian_prec": args.hessian_prec, "engine": args.engine, "damp_rel": obc_synth.DAMP_REL,
                       "l2": "per-row inverse-Hessian working set exceeds L2 (inputs larger than L2)"
                             if layer.R * layer.d * layer.d * 2 > 126e6 else "working set fits L2 (small case)",
-                      "parallelism": f"rows of one layer per GPU; {world} independent layer(s)"},
+                      "parallelism": (f"rows of ONE layer split over {world} GPUs, one all-gather of the traces before the global mask"
+                                      if sharded else f"rows of one layer per GPU; {world} independent layer(s)")},
            "stage_ms": {k: round(v, 3) for k, v in stage_sum.items()},
            "clocks": clocks, "gpu_launches": int(launches),
            "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(hW.numel() * 4 + hX.numel() * 4),
@@ -509,6 +529,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--engine", default="blocked", choices=["blocked", "streaming"],
                     help="row elimination engine: deferred block updates (default) or one pass per step")
+    ap.add_argument("--shard-rows", action="store_true",
+                    help="with --gpus N > 1: split the rows of ONE layer over the GPUs (strong scaling) instead of one layer per GPU")
     ap.add_argument("--no-compare-streaming", dest="compare_streaming", action="store_false",
                     help="skip the extra timing of the streaming engine on one wave of rows")
     args = ap.parse_args()

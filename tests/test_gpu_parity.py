@@ -362,3 +362,25 @@ def test_blocked_engine_block_sizes(threads, max_pending, d, rows):
                    gpu_codes=codes.cpu().numpy())
     finally:
         m.obc_set_engine(m.ENGINE_AUTO)
+
+
+def test_sharded_layer_driver_single_rank(obc):
+    """the row-sharded layer driver with one rank (no process group): same masks and weights as the oracle"""
+    from paper_2208_11580_b200.sharding import prune_layer_sharded
+    W, X, spec = obc_synth.make_layer("C1")
+    R, d = W.shape
+    out = prune_layer_sharded(dev(W), dev(X), (0.5, 0.75), DAMP, prec=obc.PREC_FP32)
+    torch.cuda.synchronize()
+    assert (out["row_begin"], out["row_count"]) == (0, R) and int(out["info"].item()) == 0
+    H = torch.empty(d, d, dtype=torch.float32, device="cuda")
+    obc.obc_hessian(dev(X), H, prec=obc.PREC_FP32)
+    Hinv, _ = obc.obc_hessian_inverse(H, DAMP)
+    order, loss, status, trace = run_trace(obc, dev(W), Hinv, want_trace=True)
+    res = oracle.run_rows(Hinv.cpu().numpy().astype(np.float64), W, forced=order.cpu().numpy(), want_trace=True)
+    for i, sp in enumerate((0.5, 0.75)):
+        k = obc_synth.pruned_count(R, d, sp)
+        oc, om = oracle.global_mask(loss.cpu().numpy(), order.cpu().numpy(), k)
+        assert np.array_equal(out["counts"][i].cpu().numpy(), oc) and np.array_equal(out["masks"][i].cpu().numpy(), om)
+        want = oracle.weights_from_trace(res["w_trace"], oc)
+        got = out["weights"][i].cpu().numpy()
+        assert (np.abs(got - want) / np.abs(W).max(axis=1, keepdims=True)).max() <= REL_TOL
