@@ -80,8 +80,11 @@ def inverse(H: np.ndarray, damp_rel: float):
 
 
 def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, flags=0,
-             forced=None, active0=None, want_trace=False):
+             forced=None, active0=None, want_trace=False, nm=None):
     """Algorithm 1 (mode='prune') / Algorithm 3 (mode='quant') on every row of W with the shared Hinv.
+
+    nm=(N, M): the N:M pattern of Section 3 ("N:M Sparsity", pruning only): a weight is a candidate only while its
+    block of M consecutive columns has lost fewer than M - N weights; steps defaults to d (M - N) / M.
 
     Returns a dict: order, loss, margin, best, forced_gap, round_dist, pivot_diag (rows x steps), w (rows x d final
     weights), codes (rows x d, quant only), w_trace (rows x (steps+1) x d if want_trace), status (rows).
@@ -92,6 +95,13 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
         Wd = Wd[None, :]
     rows, d = Wd.shape
     assert Hinv.shape == (d, d)
+    nm_prune, nm_block = 0, 0
+    if nm is not None:
+        n_keep, nm_block = int(nm[0]), int(nm[1])
+        assert mode == "prune" and 0 < n_keep < nm_block and d % nm_block == 0
+        nm_prune = nm_block - n_keep
+        if steps is None:
+            steps = d // nm_block * nm_prune
     steps = d if steps is None else int(steps)
     m = 1 if mode == "quant" else 0
     sc = None if scale is None else np.ascontiguousarray(np.broadcast_to(np.asarray(scale, np.float64), (rows,)))
@@ -113,7 +123,7 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
                      _p(fo, I32), _p(a0, U8), _p(out["order"], I32), _p(out["loss"], F64),
                      _p(out["margin"], F64), _p(out["best"], I32), _p(out["forced_gap"], F64),
                      _p(out["round_dist"], F64), _p(out["pivot_diag"], F64), _p(out["w_trace"], F64), _p(out["codes"], I32),
-                     _p(out["status"], I32))
+                     _p(out["status"], I32), ctypes.c_int(nm_prune), ctypes.c_int(nm_block))
     out["w"] = Wd
     return out
 
@@ -139,7 +149,8 @@ def eliminate_one_row(Hinv, w, **kw):
                         ctypes.c_double(float(kw.get("scale", 1.0))), ctypes.c_double(float(kw.get("zero", 0.0))),
                         ctypes.c_int(int(kw.get("maxq", 0))), ctypes.c_int(int(kw.get("flags", 0))),
                         _p(fo, I32), _p(a0, U8), _p(order, I32), _p(loss, F64), _p(margin, F64), _p(best, I32),
-                        _p(gap, F64), _p(rd, F64), _p(pdg, F64), _p(trace, F64), _p(codes, I32))
+                        _p(gap, F64), _p(rd, F64), _p(pdg, F64), _p(trace, F64), _p(codes, I32),
+                        ctypes.c_int(int(kw.get("nm_prune", 0))), ctypes.c_int(int(kw.get("nm_block", 0))))
     return dict(Hi=Hi, w=wd, order=order, loss=loss, margin=margin, best=best, forced_gap=gap,
                 round_dist=rd, pivot_diag=pdg, codes=codes, w_trace=trace, status=int(st))
 

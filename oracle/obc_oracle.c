@@ -107,6 +107,9 @@ static double grid_quant(double x, double scale, double zero, int maxq)
  * forced_gap[] still describe the oracle's own choice at that state.
  *   margin[t]     = (s_second - s_best) / max(s_second, tiny)   (1 when a single candidate is left)
  *   forced_gap[t] = (s_forced - s_best) / max(s_forced, tiny)
+ * N:M pattern (Section 3, "N:M Sparsity"; mode 0 only): with nm_block = M > 0 the argmin runs only over weights
+ * whose block of M consecutive columns has lost fewer than nm_prune = M - N weights so far (every block keeps
+ * exactly N non-zeros once steps = d (M - N) / M eliminations are done); nm_block = 0 switches it off.
  * With ORACLE_FLAG_OUTLIERS (Section 4, "Quantization Outliers"): if any active weight has
  * |q(w_j)-w_j| > Delta/2, the one with the largest such error is taken first (ties: lowest index).
  *
@@ -119,9 +122,11 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
                double scale, double zero, int maxq, int flags,
                const int32_t *forced, const uint8_t *active0,
                int32_t *order, double *loss, double *margin, int32_t *best, double *forced_gap,
-               double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes)
+               double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes,
+               int nm_prune, int nm_block)
 {
     const double tiny = 1e-300;
+    int32_t *blk_pruned = nm_block > 0 ? (int32_t *)calloc((size_t)(d / nm_block + 1), sizeof(int32_t)) : NULL;
     int32_t *M = (int32_t *)malloc((size_t)d * sizeof(int32_t));   /* the remaining set, ascending */
     uint8_t *in_M = (uint8_t *)calloc((size_t)d, 1);
     double *err = (double *)malloc((size_t)d * sizeof(double));
@@ -138,6 +143,7 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
             const int j = M[a];
             const double q = mode ? grid_quant(w[j], scale, zero, maxq) : 0.0;
             err[j] = q - w[j];
+            if (blk_pruned && blk_pruned[j / nm_block] >= nm_prune) continue;   /* block already at N non-zeros */
             const double s = err[j] * err[j] / Hi[(int64_t)j * d + j];
             if (b < 0 || s < sb) { b2 = b; sb2 = sb; b = j; sb = s; }
             else if (b2 < 0 || s < sb2) { b2 = j; sb2 = s; }
@@ -169,6 +175,7 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
             p = forced[t];
             if (p < 0 || p >= d || !in_M[p]) { ret = ret ? ret : 1 + t; break; }
         }
+        if (blk_pruned) blk_pruned[p / nm_block] += 1;
         const double dpp = Hi[(int64_t)p * d + p];
         if (!(dpp > 0.0) || !isfinite(dpp)) { ret = ret ? ret : 1 + t; break; }
         const double sp = err[p] * err[p] / dpp;
@@ -206,6 +213,7 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
     free(M);
     free(in_M);
     free(err);
+    free(blk_pruned);
     return ret;
 }
 
@@ -217,7 +225,8 @@ void oracle_rows(const double *Hinv, int d, int rows, double *W, int steps, int 
                  const double *scale, const double *zero, int maxq, int flags,
                  const int32_t *forced, const uint8_t *active0,
                  int32_t *order, double *loss, double *margin, int32_t *best, double *forced_gap,
-                 double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes, int32_t *status)
+                 double *round_dist, double *pivot_diag, double *w_trace, int32_t *codes, int32_t *status,
+                 int nm_prune, int nm_block)
 {
 #pragma omp parallel for schedule(dynamic, 1)
     for (int r = 0; r < rows; ++r) {
@@ -231,7 +240,7 @@ void oracle_rows(const double *Hinv, int d, int rows, double *W, int steps, int 
                                forced_gap ? forced_gap + so : NULL, round_dist ? round_dist + so : NULL,
                                pivot_diag ? pivot_diag + so : NULL,
                                w_trace ? w_trace + (int64_t)r * (steps + 1) * d : NULL,
-                               codes ? codes + (int64_t)r * d : NULL);
+                               codes ? codes + (int64_t)r * d : NULL, nm_prune, nm_block);
         free(Hi);
     }
 }

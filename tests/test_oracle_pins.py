@@ -312,3 +312,49 @@ def test_pin_k_deterministic_and_config1_fast():
     for r in (0, 13, 31):
         F = np.nonzero(mask[r])[0]
         assert np.allclose(What[r], _masked_lstsq(W[r].astype(np.float64), X_aug, list(F)), rtol=1e-6, atol=1e-10)
+
+
+@pytest.mark.parametrize("nm", [(2, 4), (4, 8), (1, 4)])
+def test_pin_nm_pattern(nm):
+    """N:M pruning (Section 3, "N:M Sparsity"): (1) every block of M consecutive weights ends with exactly N
+    non-zeros; (2) every pick is the brute-force minimiser of the true loss increase over the weights still
+    allowed (blocks that have not yet lost M - N), checked by solving each candidate's masked least-squares problem
+    directly; (3) the final weights are the masked least-squares optimum for the final support; (4) with a
+    diagonal Hessian each block simply loses its M - N smallest w_j^2 H_jj."""
+    n_keep, m = nm
+    d = 16
+    W, X, Hd, Hinv, X_aug = _problem(3, d, 80, 31 + m)
+    res = oracle.run_rows(Hinv, W, nm=nm, want_trace=True)
+    steps = d // m * (m - n_keep)
+    assert res["order"].shape[1] == steps and np.all(res["status"] == 0)
+    for r in range(W.shape[0]):
+        pruned = []
+        for t in range(steps):
+            cnt = np.bincount(np.array(pruned, dtype=np.int64) // m, minlength=d // m)
+            allowed = [j for j in range(d) if j not in pruned and cnt[j // m] < m - n_keep]
+            base = np.sum(((W[r] - res["w_trace"][r, t]) @ X_aug) ** 2)
+            inc = {}
+            for j in allowed:
+                F = [i for i in range(d) if i not in pruned and i != j]
+                v = _masked_lstsq(W[r], X_aug, F)
+                inc[j] = np.sum(((W[r] - v) @ X_aug) ** 2) - base
+            best = min(inc, key=lambda j: (inc[j], j))
+            assert best == res["order"][r, t]
+            assert np.isclose(0.5 * res["loss"][r, t], inc[best], rtol=1e-6, atol=1e-12)
+            pruned.append(int(res["order"][r, t]))
+        nz = (res["w"][r] != 0.0).reshape(d // m, m).sum(axis=1)
+        assert np.all(nz == n_keep)
+        keep = [j for j in range(d) if j not in pruned]
+        assert np.allclose(res["w"][r], _masked_lstsq(W[r], X_aug, keep), rtol=1e-8, atol=1e-11)
+    Wo, Xo = obc_synth.make_small(2, d, 40, 77, "orthogonal")
+    Ho = np.diag(np.diag(oracle.hessian(Xo, True)))
+    Hio, _ = oracle.inverse(Ho, 0.0)
+    ro = oracle.run_rows(Hio, Wo, nm=nm)
+    score = Wo.astype(np.float64) ** 2 * np.diag(Ho)
+    for r in range(2):
+        want = set()
+        for b in range(d // m):
+            idx = np.argsort(score[r, b * m:(b + 1) * m], kind="stable")[:m - n_keep] + b * m
+            want |= set(idx.tolist())
+        assert set(ro["order"][r].tolist()) == want
+        assert np.array_equal(ro["order"][r], np.array(sorted(want, key=lambda j: (score[r, j], j))))
