@@ -129,6 +129,22 @@ obc_status obc_prune_trace(const float *W, int ldw, int d_row, int d_col, int ro
                            int32_t *order, float *loss, float *w_trace, int32_t *row_status,
                            void *ws, size_t ws_bytes, obc_stream stream);
 
+/* Section 3, "N:M Sparsity": Algorithm 1 with the argmin restricted to weights whose block of m_block consecutive
+ * columns has lost fewer than m_block - n_keep weights so far; after d_col * (m_block - n_keep) / m_block
+ * eliminations every block keeps exactly n_keep non-zeros, and no global step is needed (all rows have the same
+ * sparsity).  (The paper's sentence counts "< N pruned weights", which equals m_block - n_keep for its 2:4 and 4:8
+ * patterns; the count used here is the general one.)
+ *   m_block in {2, 4, 8, 16, 32}, 0 < n_keep < m_block, d_col a multiple of m_block.
+ *   order, loss: d_row x d_col as in obc_prune_trace, the first d_col*(m_block-n_keep)/m_block entries of a row
+ *                are written; nullable.
+ *   W_out : d_row x d_col FP32 (ldwo): the compensated weights, 0 at pruned positions.
+ *   mask  : nullable d_row x d_col uint8, 1 = kept.
+ * Always runs on the BLOCKED engine.  Workspace: obc_workspace_bytes(OBC_OP_PRUNE_TRACE, row_count, d_col, 0). */
+obc_status obc_prune_nm(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                        const float *Hinv, int ldhi, int n_keep, int m_block,
+                        int32_t *order, float *loss, float *W_out, int ldwo, uint8_t *mask, int32_t *row_status,
+                        void *ws, size_t ws_bytes, obc_stream stream);
+
 /* Algorithm 2 (appendix, "ExactOBS Global Step"): repeatedly prune, across all rows, the weight whose
  * next recorded loss is smallest (ties: lowest row), k times.  k is a count, 0 <= k <= d_row*d_col.
  *   counts: d_row int32, weights pruned per row;  mask: d_row x d_col uint8, 0 at order[r][t], t < counts[r].

@@ -19,7 +19,7 @@ FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace",
+    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -63,6 +63,9 @@ def load_library():
     lib.obc_hessian_inverse.argtypes = [vp, c_int, c_int, c_f, vp, c_int, vp, vp, c_sz, vp]
     lib.obc_prune_trace.restype = c_int
     lib.obc_prune_trace.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+    lib.obc_prune_nm.restype = c_int
+    lib.obc_prune_nm.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, c_int, vp, vp, vp, c_int, vp, vp,
+                                 vp, c_sz, vp]
     lib.obc_select_global_mask.restype = c_int
     lib.obc_select_global_mask.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp, c_sz, vp]
     lib.obc_select_global_mask_static.restype = c_int
@@ -178,6 +181,20 @@ def obc_prune_trace(W, Hinv, order, loss, row_status, steps=None, w_trace=None, 
     _raise(load_library().obc_prune_trace(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), steps,
                                           _ptr(order), _ptr(loss), _ptr(w_trace), _ptr(row_status), _ptr(ws), nb,
                                           _stream(stream)), "obc_prune_trace")
+
+
+def obc_prune_nm(W, Hinv, n_keep, m_block, W_out, row_status, order=None, loss=None, mask=None, row_begin=0,
+                 row_count=None, ws=None, stream=None):
+    """N:M pruning of rows [row_begin, row_begin+row_count): every block of m_block columns keeps n_keep weights."""
+    _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(W_out, torch.float32, "W_out")
+    _check(row_status, torch.int32, "row_status"); _check(order, torch.int32, "order"); _check(loss, torch.float32, "loss")
+    _check(mask, torch.uint8, "mask")
+    R, d = W.shape
+    row_count = R - row_begin if row_count is None else row_count
+    ws, nb = _workspace(ws, OP_PRUNE_TRACE, row_count, d, 0, W.device, "obc_prune_nm")
+    _raise(load_library().obc_prune_nm(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), int(n_keep),
+                                       int(m_block), _ptr(order), _ptr(loss), _ptr(W_out), _ld(W_out), _ptr(mask),
+                                       _ptr(row_status), _ptr(ws), nb, _stream(stream)), "obc_prune_nm")
 
 
 def obc_select_global_mask(loss, order, k, counts, mask, ws=None, stream=None):

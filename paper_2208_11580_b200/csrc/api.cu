@@ -130,6 +130,21 @@ obc_status obc_prune_trace(const float* W, int ldw, int d_row, int d_col, int ro
                               row_status, ws, ws_bytes, (cudaStream_t)stream);
 }
 
+obc_status obc_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                        const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
+                        float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
+                        obc_stream stream) {
+    if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (!mat_ok(W_out, ldwo, d_col) || !row_status) return OBC_ERR_INVALID_ARG;
+    if (m_block != 2 && m_block != 4 && m_block != 8 && m_block != 16 && m_block != 32) return OBC_ERR_INVALID_ARG;
+    if (n_keep <= 0 || n_keep >= m_block || d_col % m_block != 0) return OBC_ERR_INVALID_ARG;
+    if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    return engine_prune_nm(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, n_keep, m_block, order, loss, W_out,
+                           ldwo, mask, row_status, ws, ws_bytes, (cudaStream_t)stream);
+}
+
 obc_status obc_select_global_mask(const float* loss, const int32_t* order, int d_row, int d_col, int64_t k,
                                   int32_t* counts, uint8_t* mask, void* ws, size_t ws_bytes, obc_stream stream) {
     if (d_row <= 0 || d_col <= 0 || !loss || !order || !counts || !mask) return OBC_ERR_INVALID_ARG;

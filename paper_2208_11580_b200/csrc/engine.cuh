@@ -26,6 +26,9 @@ struct EngineArgs {
     int cap;                              // d rounded up to a multiple of 4
     int panel_floats;                     // blocked engine: floats of shared memory for the pending vectors
     int max_pending;                      // blocked engine: upper limit on deferred updates (1..64)
+    int nm_prune; int nm_lg;              // blocked engine, N:M pattern: at most nm_prune eliminations per block of
+                                          // 2^nm_lg consecutive columns (nm_prune = 0: no pattern)
+    uint8_t* mask;                        // blocked engine, nullable: d_row x d mask, 0 at eliminated columns
 };
 
 struct Bcast {                            // block-wide broadcast values, written by one thread

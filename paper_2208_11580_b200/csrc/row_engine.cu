@@ -444,6 +444,20 @@ obc_status engine_prune_trace(const float* W, int ldw, int d_row, int d_col, int
     return engine_launch(a, ws, ws_bytes, stream);
 }
 
+obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                           const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
+                           float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
+                           cudaStream_t stream) {
+    (void)d_row;
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    a.mode = MODE_PRUNE; a.steps = d_col / m_block * (m_block - n_keep); a.order = order; a.loss = loss;
+    a.trace_steps = a.steps; a.W_out = W_out; a.ldwo = ldwo; a.mask = mask;
+    a.nm_prune = m_block - n_keep;
+    a.nm_lg = 0;
+    while ((1 << a.nm_lg) < m_block) ++a.nm_lg;
+    return blocked_engine_launch(a, ws, ws_bytes, stream);      // the pattern is built into the blocked engine only
+}
+
 obc_status engine_replay(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                          const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts, float* W_out,
                          int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {

@@ -40,8 +40,11 @@ constexpr int BLK_OFF_CM = 2304;              // uint32 colmask[160]: bit j set 
 constexpr int BLK_OFF_RF = 2944;              // float rf[64]  min/max reduction of the compound grid
 constexpr int BLK_FIXED = 3200;
 
-__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull) {
-    return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0);
+// Per-row state in shared memory: wd, dg (FP64), perm (int32), srcm (uint16); optional: the row in original
+// order (weight trace), one byte per block of the N:M pattern.
+__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm = false) {
+    return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0) +
+           (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0);
 }
 static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
 
@@ -131,14 +134,25 @@ __device__ __forceinline__ float score_estimate(double w, double dgv, bool quant
 }
 
 // Estimates of all own slots from the state arrays (NaN for dead or unused slots).
+// N:M pattern: blkcnt (nullable) holds per block of 2^nm_lg original columns the number of weights eliminated so
+// far; a slot whose block has reached nm_prune is no candidate (NaN estimate).  cntw receives the counts of the
+// own slots' blocks, one byte per slot, which the update phase then keeps current in registers.
 template <int NT, int KMAX>
 __device__ __forceinline__ void estimate_own(float (&sa)[KMAX], const double* wd, const double* dg, const int* perm,
-                                             int m0, bool quant, double sc, double isc, double ze, double mq) {
+                                             int m0, bool quant, double sc, double isc, double ze, double mq,
+                                             const unsigned char* blkcnt, int nm_lg, int nm_prune,
+                                             unsigned (&cntw)[KMAX / 4]) {
+#pragma unroll
+    for (int g = 0; g < KMAX / 4; ++g) cntw[g] = 0u;
 #pragma unroll
     for (int k = 0; k < KMAX; ++k) {
         const int j = own_slot<NT>(k);
         sa[k] = CUDART_NAN_F;
-        if (j < m0 && perm[j] >= 0) sa[k] = score_estimate(wd[j], dg[j], quant, sc, isc, ze, mq);
+        if (j < m0 && perm[j] >= 0) {
+            unsigned c = 0u;
+            if (blkcnt) { c = blkcnt[perm[j] >> nm_lg]; cntw[k >> 2] |= c << (8 * (k & 3)); }
+            if (!blkcnt || (int)c < nm_prune) sa[k] = score_estimate(wd[j], dg[j], quant, sc, isc, ze, mq);
+        }
     }
 }
 
@@ -288,7 +302,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     unsigned short* srcm = reinterpret_cast<unsigned short*>(perm + cap);
     const bool has_wfull = a.w_trace != nullptr;
     float* wfull = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, false));
-    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull));
+    const bool has_nm = a.nm_prune > 0;                         // N:M pattern: at most nm_prune eliminations per block
+    const int nm_lg = a.nm_lg, nm_prune = a.nm_prune;
+    unsigned char* blkcnt = reinterpret_cast<unsigned char*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull));
+    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm));
     // tail views (step-by-step phase in shared memory) share the panel's space
     const int msr = (ms + 3) & ~3;
     float* tv = panel;
@@ -322,7 +339,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             srcm[j] = (unsigned short)j;
             if (has_wfull) wfull[j] = w;
             if (a.codes) a.codes[(size_t)r * d + j] = -1;
+            if (a.mask) a.mask[(size_t)r * d + j] = 1;
         }
+        if (has_nm) for (int b = tid; b < (d >> nm_lg); b += NT) blkcnt[b] = 0;
         for (int j = d + tid; j < cap; j += NT) perm[j] = -1;
         for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
         if (tid == 0) {
@@ -355,6 +374,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         int s = 0;
         bool failed = false;
         float sa[KMAX];                  // score estimates of the own slots, kept up to date by the update phase
+        unsigned cntw[KMAX / 4];         // N:M: eliminations so far in the block of each own slot (one byte per slot)
+#pragma unroll
+        for (int g = 0; g < KMAX / 4; ++g) cntw[g] = 0u;
         bool sa_valid = false;
         double gisc = 1.0 / gsc;
         for (; s < total; ++s) {
@@ -398,6 +420,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     sa_valid = false;
 #pragma unroll
                     for (int k = 0; k < KMAX; ++k) sa[k] = CUDART_NAN_F;      // slots changed hands: not carried over
+#pragma unroll
+                    for (int g = 0; g < KMAX / 4; ++g) cntw[g] = 0u;
                     ldz = (m0 + 15) & ~15;
                     bcur = min(a.max_pending, a.panel_floats / ldz);
                     __syncthreads();
@@ -451,7 +475,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 }
             } else {
                 if (!sa_valid || tail || outliers)
-                    estimate_own<NT, KMAX>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq);
+                    estimate_own<NT, KMAX>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq, has_nm ? blkcnt : nullptr,
+                                           nm_lg, nm_prune, cntw);
                 thread_best<NT, KMAX>(sa, wd, dg, perm, q_now, outliers, gsc, gisc, gze, gmq, &key, &cs, &cslot);
             }
             const Records rec = rec_view(scratch, s & 1);
@@ -517,6 +542,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 for (int g = 0; g < KMAX / 4; ++g) {
                     const int jb = own_slot<NT>(4 * g);
                     if (jb >= m0) continue;
+                    const int4 pm = *reinterpret_cast<const int4*>(perm + jb);
+                    const int pq[4] = {pm.x, pm.y, pm.z, pm.w};
                     float zv[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
@@ -524,14 +551,22 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         zv[q] = 0.f;
                         sa[k] = CUDART_NAN_F;
                         if (!((live >> k) & 1u)) continue;
-                        if (j == p) { perm[j] = -1; continue; }
+                        if (j == p) {
+                            perm[j] = -1;
+                            if (has_nm) blkcnt[op >> nm_lg] += 1;      // read again only behind a barrier
+                            continue;
+                        }
                         const float vj = c[k] - corr[k];
                         const double nw = wd[j] - f * (double)vj;
                         const double nd = dg[j] - (double)vj * (double)vj * idpp;
                         wd[j] = nw; dg[j] = nd;
                         zv[q] = vj * rs;
                         if (est_next) sa[k] = score_estimate(nw, nd, q_next, gsc, gisc, gze, gmq);
-                        if (has_wfull) wfull[perm[j]] = (float)nw;
+                        if (has_nm) {
+                            if ((pq[q] >> nm_lg) == (op >> nm_lg)) cntw[g] += 1u << (8 * q);
+                            if ((int)((cntw[g] >> (8 * q)) & 0xFFu) >= nm_prune) sa[k] = CUDART_NAN_F;
+                        }
+                        if (has_wfull) wfull[pq[q]] = (float)nw;
                     }
                     *reinterpret_cast<float4*>(zb + jb) = make_float4(zv[0], zv[1], zv[2], zv[3]);
                 }
@@ -540,6 +575,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     pv[nb] = p;
                     if (has_wfull) wfull[op] = (float)qp;
                     if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)qp;
+                    if (a.mask) a.mask[(size_t)r * d + op] = 0;
                     if (!forced) {
                         const int t = s - n_forced;
                         if (a.order) a.order[(size_t)r * d + t] = op;
@@ -577,6 +613,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         if (j == last) { perm[p] = oj; tv[p] = vj; tlr[p] = tlr[last]; }
                     }
                     if (tid == 0) {
+                        if (has_nm) blkcnt[op >> nm_lg] += 1;
+                        if (a.mask) a.mask[(size_t)r * d + op] = 0;
                         if (has_wfull) wfull[op] = (float)qp;
                         if (a.W_out) a.W_out[(size_t)r * a.ldwo + op] = (float)qp;
                         if (!forced) {
@@ -632,7 +670,7 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 
 // Threads per block and blocks per SM by row length: short rows are bound by the latency of a step, so
 // several of them share an SM; long rows need the shared memory for pending vectors.
-static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out) {
+static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false) {
     const int cap = (d + 3) & ~3;
     int nt = engine_threads_choice();
     if (nt != 128 && nt != 256 && nt != 512) nt = d <= 1024 ? 128 : (d <= 2048 ? 256 : 512);
@@ -645,7 +683,7 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out) {
     const size_t sm_total = (size_t)di.smem_optin + 1024;
     size_t share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
     if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
-    const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull);
+    const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull, nm);
     const size_t min_panel = (size_t)4 * ((cap + 15) & ~15);
     while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
         p.per_sm >>= 1;
@@ -699,7 +737,7 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     a.cap = (a.d + 3) & ~3;
     if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     BlkPlan p;
-    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p)) return OBC_ERR_UNSUPPORTED;
+    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0)) return OBC_ERR_UNSUPPORTED;
     a.ms = p.ms;
     a.panel_floats = p.panel_floats;
     int mp = engine_pending_choice();

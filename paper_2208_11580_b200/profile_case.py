@@ -24,7 +24,7 @@ def main():
     ap.add_argument("--d", type=int, default=1152)
     ap.add_argument("--rows", type=int, default=148)
     ap.add_argument("--n", type=int, default=0)
-    ap.add_argument("--mode", default="prune", choices=["prune", "quant", "hessian"])
+    ap.add_argument("--mode", default="prune", choices=["prune", "quant", "nm24", "hessian"])
     ap.add_argument("--prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
     ap.add_argument("--repeat", type=int, default=2)
     ap.add_argument("--engine", default="auto", choices=["auto", "streaming", "blocked"])
@@ -58,6 +58,8 @@ def main():
     loss = torch.zeros(R, d, dtype=torch.float32, device="cuda")
     status = torch.zeros(R, dtype=torch.int32, device="cuda")
     ws = torch.empty(obc.obc_workspace_bytes(obc.OP_PRUNE_TRACE, R, d), dtype=torch.uint8, device="cuda")
+    if a.mode == "nm24":
+        Wq = torch.zeros(R, d, dtype=torch.float32, device="cuda")
     if a.mode == "quant":
         scale = torch.zeros(R, dtype=torch.float32, device="cuda")
         zero = torch.zeros(R, dtype=torch.float32, device="cuda")
@@ -70,6 +72,8 @@ def main():
         e0.record()
         if a.mode == "prune":
             obc.obc_prune_trace(Wd, Hinv, order, loss, status, ws=ws)
+        elif a.mode == "nm24":
+            obc.obc_prune_nm(Wd, Hinv, 2, 4, Wq, status, order=order, loss=loss, ws=ws)
         else:
             obc.obc_quantize(Wd, Hinv, scale, zero, 4, False, Wq, codes, status, ws=ws)
         e1.record()

@@ -16,7 +16,7 @@ ROUND_TOL = 1e-4       # integer codes may differ only if x/Delta is this close 
 
 
 def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", scale=None, zero=None, maxq=0,
-               flags=0, gpu_codes=None, gpu_trace=None, steps=None, active0=None):
+               flags=0, gpu_codes=None, gpu_trace=None, steps=None, active0=None, nm=None):
     """Compare GPU results for a set of rows with the oracle fed the same FP32 Hinv / W.
     Returns a dict of statistics; raises AssertionError on a parity violation."""
     Hinv = np.asarray(Hinv32, dtype=np.float64)
@@ -25,7 +25,7 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
     steps = d if steps is None else steps
     gpu_order = np.asarray(gpu_order)[:, :steps]
     res = oracle.run_rows(Hinv, W, steps=steps, mode=mode, scale=scale, zero=zero, maxq=maxq, flags=flags,
-                          forced=gpu_order, active0=active0, want_trace=gpu_trace is not None)
+                          forced=gpu_order, active0=active0, want_trace=gpu_trace is not None, nm=nm)
     assert np.all(res["status"] == 0), f"oracle rejected the GPU order: {res['status']}"
     differ = res["best"] != gpu_order
     gap = res["forced_gap"]

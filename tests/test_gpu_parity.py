@@ -384,3 +384,37 @@ def test_sharded_layer_driver_single_rank(obc):
         want = oracle.weights_from_trace(res["w_trace"], oc)
         got = out["weights"][i].cpu().numpy()
         assert (np.abs(got - want) / np.abs(W).max(axis=1, keepdims=True)).max() <= REL_TOL
+
+
+@pytest.mark.parametrize("threads,max_pending", [(0, 0), (128, 3), (512, 5)])
+@pytest.mark.parametrize("nm", [(2, 4), (4, 8), (1, 4), (1, 2)])
+@pytest.mark.parametrize("d,rows", [(16, 3), (304, 4), (640, 3)])
+def test_prune_nm_against_oracle(nm, d, rows, threads, max_pending):
+    """N:M pruning (Section 3, "N:M Sparsity"): picks, losses and compensated weights against the oracle, the mask
+    keeps exactly N weights in every block of M"""
+    import paper_2208_11580_b200 as m
+    m.load_library()
+    n_keep, mb = nm
+    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
+    try:
+        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1200 + d + mb, "relu")
+        H = oracle.hessian(X).astype(np.float32)
+        Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
+        Wd = dev(W)
+        steps = d // mb * (mb - n_keep)
+        order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
+        loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
+        Wout = torch.full((rows, d), 9.0, dtype=torch.float32, device="cuda")
+        mask = torch.full((rows, d), 9, dtype=torch.uint8, device="cuda")
+        rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+        m.obc_prune_nm(Wd, Hinv, n_keep, mb, Wout, rs, order=order, loss=loss, mask=mask)
+        torch.cuda.synchronize()
+        assert int(rs.abs().sum()) == 0
+        o, mk, wo = order.cpu().numpy(), mask.cpu().numpy(), Wout.cpu().numpy()
+        assert np.all(o[:, steps:] == -7) and np.all(mk.reshape(rows, d // mb, mb).sum(axis=2) == n_keep)
+        assert np.all(wo[mk == 0] == 0.0)
+        for r in range(rows):
+            assert set(np.nonzero(mk[r] == 0)[0].tolist()) == set(o[r, :steps].tolist())
+        check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), gpu_w=wo, steps=steps, nm=nm)
+    finally:
+        m.obc_set_engine(m.ENGINE_AUTO)
