@@ -4,7 +4,7 @@
 // One d^3 job per layer, carried in FP64 so that the FP32 result is correctly rounded to well below the
 // elimination engine's own error:  A = H + lambda I  ->  blocked right-looking Cholesky A = L L^T
 // (48-wide panels; diagonal block factored and inverted by one CTA, panel solved against the inverted
-// diagonal block, trailing matrix updated by a tiled FP64 GEMM)  ->  blocked inverse of L  ->
+// diagonal block, trailing matrix updated by a tiled FP64 GEMM)  ->  inverse of L by block doubling  ->
 // Hinv = L^-T L^-1 (lower tiles) -> mirrored, exactly symmetric FP32 output.
 #include "common.cuh"
 
@@ -18,24 +18,20 @@ constexpr int GK = 16;
 // stored NxK.  lower_only: skip tiles strictly above the diagonal (M == N outputs that are symmetric).
 // k_lo_from_tile: the product only needs k >= max(first row, first column) of the tile (L^-T L^-1).
 template <bool TA, bool TB>
-__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double alpha, const double* __restrict__ A, int lda,
-                                                    const double* __restrict__ B, int ldb, double beta,
-                                                    double* __restrict__ C, int ldc, int lower_only, int k_lo_from_tile) {
-    const int bm = blockIdx.y * GT, bn = blockIdx.x * GT;
-    if (lower_only && bn > bm + GT - 1) return;
+__device__ __forceinline__ void dgemm_tile(int M, int N, double alpha, const double* __restrict__ A, int lda,
+                                           const double* __restrict__ B, int ldb, double beta, double* __restrict__ C,
+                                           int ldc, int bm, int bn, int k_begin, int k_end) {
     __shared__ double As[GK][GT + 1];
     __shared__ double Bs[GK][GT + 1];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     double acc[4][4] = {};
-    int k0 = 0;
-    if (k_lo_from_tile) k0 = (max(bm, bn) / GK) * GK;
-    for (; k0 < K; k0 += GK) {
+    for (int k0 = k_begin; k0 < k_end; k0 += GK) {
         for (int e = tid; e < GT * GK; e += 256) {
             int i, k;
             if (TA) { i = e % GT; k = e / GT; } else { k = e % GK; i = e / GK; }
             const int gi = bm + i, gk = k0 + k;
             double v = 0.0;
-            if (gi < M && gk < K) v = TA ? A[(size_t)gk * lda + gi] : A[(size_t)gi * lda + gk];
+            if (gi < M && gk < k_end) v = TA ? A[(size_t)gk * lda + gi] : A[(size_t)gi * lda + gk];
             As[k][i] = v;
         }
         for (int e = tid; e < GT * GK; e += 256) {
@@ -43,7 +39,7 @@ __global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double 
             if (TB) { k = e % GK; j = e / GK; } else { j = e % GT; k = e / GT; }
             const int gj = bn + j, gk = k0 + k;
             double v = 0.0;
-            if (gj < N && gk < K) v = TB ? B[(size_t)gj * ldb + gk] : B[(size_t)gk * ldb + gj];
+            if (gj < N && gk < k_end) v = TB ? B[(size_t)gj * ldb + gk] : B[(size_t)gk * ldb + gj];
             Bs[k][j] = v;
         }
         __syncthreads();
@@ -71,6 +67,38 @@ __global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double 
                 *c = (beta == 0.0 ? 0.0 : beta * *c) + alpha * acc[i][j];
             }
         }
+}
+
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double alpha, const double* __restrict__ A, int lda,
+                                                    const double* __restrict__ B, int ldb, double beta,
+                                                    double* __restrict__ C, int ldc, int lower_only, int k_lo_from_tile) {
+    const int bm = blockIdx.y * GT, bn = blockIdx.x * GT;
+    if (lower_only && bn > bm + GT - 1) return;
+    int k0 = 0;
+    if (k_lo_from_tile) k0 = (max(bm, bn) / GK) * GK;
+    dgemm_tile<TA, TB>(M, N, alpha, A, lda, B, ldb, beta, C, ldc, bm, bn, k0, K);
+}
+
+// One level of the recursive inverse of the lower-triangular factor.  With the inverses of the diagonal blocks of
+// size s known, the diagonal blocks of size 2s follow from
+//      inv([[L11, 0], [L21, L22]]) = [[X11, 0], [-X22 L21 X11, X22]] ,   X11 = inv(L11), X22 = inv(L22),
+// for all pairs of blocks at once (blockIdx.z = pair; the last pair may be short or lack its second block).
+// stage 0:  T = L21 * X11  (into the scratch matrix at the position of L21);  stage 1:  X21 = -X22 * T.
+// X11 and X22 are lower triangular, which bounds the k range of every tile.
+__global__ void __launch_bounds__(256) trinv_level_kernel(const double* __restrict__ L, double* __restrict__ X,
+                                                          double* __restrict__ T, int d, int s, int stage) {
+    const int lo = blockIdx.z * 2 * s;
+    const int s1 = min(s, d - lo);
+    const int s2 = min(s, d - lo - s);
+    if (s2 <= 0) return;
+    const int bm = blockIdx.y * GT, bn = blockIdx.x * GT;
+    if (bm >= s2 || bn >= s1) return;
+    const size_t o21 = (size_t)(lo + s) * d + lo, o11 = (size_t)lo * d + lo, o22 = (size_t)(lo + s) * d + lo + s;
+    if (stage == 0)      // (T)[i][j] = sum_{k >= j} L21[i][k] X11[k][j]
+        dgemm_tile<false, false>(s2, s1, 1.0, L + o21, d, X + o11, d, 0.0, T + o21, d, bm, bn, (bn / GK) * GK, s1);
+    else                 // X21[i][j] = -sum_{k <= i} X22[i][k] T[k][j]
+        dgemm_tile<false, false>(s2, s1, -1.0, X + o22, d, T + o21, d, 0.0, X + o21, d, bm, bn, 0, min(s2, bm + GT));
 }
 
 template <bool TA, bool TB>
@@ -199,7 +227,7 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
     double* A = reinterpret_cast<double*>(p); p += mat;
     double* Li = reinterpret_cast<double*>(p); p += mat;
     double* C = reinterpret_cast<double*>(p); p += mat;
-    double* T = reinterpret_cast<double*>(p); p += round_up((size_t)NB * d * sizeof(double), 256);
+    p += round_up((size_t)NB * d * sizeof(double), 256);         // (reserved)
     double* lambda = reinterpret_cast<double*>(p);
 
     damp_kernel<<<1, 256, 0, s>>>(H, ldh, d, damp_rel, lambda, info);
@@ -219,11 +247,14 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
             dgemm<false, true>(s, below, below, nb, -1.0, P, d, P, d, 1.0, A + (size_t)(k0 + nb) * d + k0 + nb, d, 1, 0);
         }
     }
-    // blocked inverse of L: Li[i,0:i] = -Li_ii * (L[i,0:i] * Li[0:i,0:i])
-    for (int i0 = NB; i0 < d; i0 += NB) {
-        const int nb = d - i0 < NB ? d - i0 : NB;
-        dgemm<false, false>(s, nb, i0, i0, 1.0, A + (size_t)i0 * d, d, Li, d, 0.0, T, d);
-        dgemm<false, false>(s, nb, i0, nb, -1.0, Li + (size_t)i0 * d + i0, d, T, d, 0.0, Li + (size_t)i0 * d, d);
+    // inverse of L by block doubling: the diagonal NB-blocks of Li are known from the factorisation; each level
+    // fills the off-diagonal halves of the diagonal blocks of twice the size, all pairs in one launch (C = scratch)
+    for (int bs = NB; bs < d; bs *= 2) {
+        const int pairs = (d + 2 * bs - 1) / (2 * bs);
+        dim3 grid((bs + GT - 1) / GT, (bs + GT - 1) / GT, pairs);
+        trinv_level_kernel<<<grid, 256, 0, s>>>(A, Li, C, d, bs, 0);
+        trinv_level_kernel<<<grid, 256, 0, s>>>(A, Li, C, d, bs, 1);
+        count_launch(2);
     }
     // C = Li^T Li on the lower tiles, then mirror into FP32
     dgemm<true, false>(s, d, d, d, 1.0, Li, d, Li, d, 0.0, C, d, 1, 1);
