@@ -36,7 +36,7 @@ constexpr int BLK_OFF_BC = 1280;              // Bcast (grid parameters, flush b
 constexpr int BLK_OFF_PV = 1536;              // int pv[64]   slots eliminated since the last flush
 constexpr int BLK_OFF_HL = 1792;              // int hl[64]   holes (dead slots below the new size)
 constexpr int BLK_OFF_MV = 2048;              // int mv[64]   live slots that move into the holes
-constexpr int BLK_OFF_CM = 2304;              // uint32 colmask[160]: bit j set = column j is a hole
+constexpr int BLK_OFF_CM = 2304;
 constexpr int BLK_OFF_RF = 2944;              // float rf[64]  min/max reduction of the compound grid
 constexpr int BLK_FIXED = 3200;
 
@@ -124,20 +124,32 @@ __device__ __forceinline__ Pick block_pick(unsigned key, double s, int slot, int
 template <int NT>
 __device__ __forceinline__ int own_slot(int k) { return (k >> 2) * (4 * NT) + (threadIdx.x << 2) + (k & 3); }
 
+// err = q(w) - w on the row's grid.  Kept out of line: it is reached once per slot and step in the OBQ kernels,
+// and inlining it at every use multiplies the code size of a kernel whose instruction footprint already matters
+// (several rows in different phases share one SM's instruction cache).
+__device__ __noinline__ double grid_error(double w, double sc, double isc, double ze, double mq) {
+    double code;
+    return grid_q_fast(w, sc, isc, ze, mq, &code) - w;
+}
+
 // FP32 estimate of the score of a slot (relative error of a few 1e-7): it only screens candidates, the slots
 // within 1e-4 of the thread's best estimate are scored again with the FP64 division.
+template <bool Q>
 __device__ __forceinline__ float score_estimate(double w, double dgv, bool quant, double sc, double isc, double ze,
                                                 double mq) {
-    double err = -w, code;
-    if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
-    return __fdividef(__double2float_rn(err * err), __double2float_rn(dgv));
+    if (Q && quant) {
+        const double err = grid_error(w, sc, isc, ze, mq);
+        return __fdividef(__double2float_rn(err * err), __double2float_rn(dgv));
+    }
+    const float wf = __double2float_rn(w);
+    return __fdividef(wf * wf, __double2float_rn(dgv));
 }
 
 // Estimates of all own slots from the state arrays (NaN for dead or unused slots).
 // N:M pattern: blkcnt (nullable) holds per block of 2^nm_lg original columns the number of weights eliminated so
 // far; a slot whose block has reached nm_prune is no candidate (NaN estimate).  cntw receives the counts of the
 // own slots' blocks, one byte per slot, which the update phase then keeps current in registers.
-template <int NT, int KMAX>
+template <int NT, int KMAX, bool Q>
 __device__ __forceinline__ void estimate_own(float (&sa)[KMAX], const double* wd, const double* dg, const int* perm,
                                              int m0, bool quant, double sc, double isc, double ze, double mq,
                                              const unsigned char* blkcnt, int nm_lg, int nm_prune,
@@ -151,16 +163,18 @@ __device__ __forceinline__ void estimate_own(float (&sa)[KMAX], const double* wd
         if (j < m0 && perm[j] >= 0) {
             unsigned c = 0u;
             if (blkcnt) { c = blkcnt[perm[j] >> nm_lg]; cntw[k >> 2] |= c << (8 * (k & 3)); }
-            if (!blkcnt || (int)c < nm_prune) sa[k] = score_estimate(wd[j], dg[j], quant, sc, isc, ze, mq);
+            if (!blkcnt || (int)c < nm_prune) sa[k] = score_estimate<Q>(wd[j], dg[j], quant, sc, isc, ze, mq);
         }
     }
 }
 
 // The thread's best live slot among its own by (score, original index), given the estimates: only the slots
 // within 1e-4 of the thread's best estimate take the FP64 division, so the result (ties included) is the
-// exact FP64 choice.  With the outlier rule (Section 4, "Quantization Outliers") a slot whose error exceeds
-// Delta/2 wins by largest error; such candidates get negative scores, below every regular one.
-template <int NT, int KMAX>
+// exact FP64 choice.  The candidates are first collected in a bit mask and then scored in one loop, so the
+// exact scoring exists once in the code and the lanes of a warp take it together.
+// With the outlier rule (Section 4, "Quantization Outliers") a slot whose error exceeds Delta/2 wins by
+// largest error; such candidates get negative scores, below every regular one.
+template <int NT, int KMAX, bool Q>
 __device__ __forceinline__ void thread_best(const float (&sa)[KMAX], const double* wd, const double* dg,
                                             const int* perm, bool quant, bool outliers, double sc, double isc,
                                             double ze, double mq, unsigned* key, double* s_out, int* slot_out) {
@@ -168,30 +182,35 @@ __device__ __forceinline__ void thread_best(const float (&sa)[KMAX], const doubl
 #pragma unroll
     for (int k = 0; k < KMAX; ++k) smin = fminf(smin, sa[k]);           // fminf ignores NaN estimates
     const float thr = smin + 1e-4f * fabsf(smin);
-    double bs = CUDART_INF, oe = -1.0;
-    int bo = 0x7fffffff, bslot = -1, oo = 0x7fffffff, oslot = -1;
+    unsigned cand = 0u, valid = 0u;
 #pragma unroll
     for (int k = 0; k < KMAX; ++k) {
-        const bool cand = sa[k] <= thr || sa[k] == smin;                 // false for NaN estimates
-        if (cand || (outliers && sa[k] == sa[k])) {
-            const int j = own_slot<NT>(k);
-            const double w = wd[j];
-            double err = -w, code;
-            if (quant) err = grid_q_fast(w, sc, isc, ze, mq, &code) - w;
-            const int o = perm[j];
-            if (cand) {
-                const double s = err * err / dg[j];
-                if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
-            }
-            if (outliers) {
-                const double a = fabs(err);
-                if (a > 0.5 * sc && (a > oe || (a == oe && o < oo))) { oe = a; oo = o; oslot = j; }
-            }
+        if (sa[k] <= thr || sa[k] == smin) cand |= 1u << k;             // false for NaN estimates
+        if (sa[k] == sa[k]) valid |= 1u << k;
+    }
+    double bs = CUDART_INF, oe = -1.0;
+    int bo = 0x7fffffff, bslot = -1, oo = 0x7fffffff, oslot = -1;
+    unsigned todo = (Q && outliers) ? valid : cand;
+    while (todo) {
+        const int k = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int j = own_slot<NT>(k);
+        const double w = wd[j];
+        double err = -w;
+        if (Q && quant) err = grid_error(w, sc, isc, ze, mq);
+        const int o = perm[j];
+        if ((cand >> k) & 1u) {
+            const double s = err * err / dg[j];
+            if (key_less(s, o, bs, bo)) { bs = s; bo = o; bslot = j; }
+        }
+        if (Q && outliers) {
+            const double a = fabs(err);
+            if (a > 0.5 * sc && (a > oe || (a == oe && o < oo))) { oe = a; oo = o; oslot = j; }
         }
     }
     *key = KEY_NONE; *s_out = bs; *slot_out = bslot;
     if (bslot >= 0) *key = float_key(__double2float_rn(bs));
-    if (outliers && oslot >= 0) { *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe)); }
+    if (Q && outliers && oslot >= 0) { *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe)); }
 }
 
 // Applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts
@@ -283,7 +302,8 @@ __device__ __forceinline__ void blk_pass_shared(float* S, int lds, int mp, int p
     }
 }
 
-template <int NT, int KMAX>
+// Q = the kernel contains the OBQ code (modes QUANT and REPLAY_QUANT); the pruning kernels are built without it.
+template <int NT, int KMAX, bool Q>
 __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
     extern __shared__ __align__(16) char smem[];
     constexpr int NW = NT / 32;
@@ -294,8 +314,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     int* pv = reinterpret_cast<int*>(smem + BLK_OFF_PV);
     int* hl = reinterpret_cast<int*>(smem + BLK_OFF_HL);
     int* mv = reinterpret_cast<int*>(smem + BLK_OFF_MV);
-    uint32_t* colmask = reinterpret_cast<uint32_t*>(smem + BLK_OFF_CM);
     float* rf = reinterpret_cast<float*>(smem + BLK_OFF_RF);
+    uint32_t* colmask = reinterpret_cast<uint32_t*>(smem + BLK_OFF_CM);
     double* wd = reinterpret_cast<double*>(smem + BLK_FIXED);
     double* dg = wd + cap;
     int* perm = reinterpret_cast<int*>(dg + cap);
@@ -322,13 +342,13 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         bool quant = false;
         if (a.mode == MODE_PRUNE) { n_free = a.steps; }
         else if (a.mode == MODE_REPLAY) { n_forced = a.forced_counts[r]; }
-        else if (a.mode == MODE_QUANT) { n_free = d; quant = true; }
-        else { n_forced = a.forced_counts[r]; n_free = d - n_forced; quant = true; }
+        else if (a.mode == MODE_QUANT) { n_free = d; quant = Q; }
+        else { n_forced = a.forced_counts[r]; n_free = d - n_forced; quant = Q; }
         if (n_forced < 0) n_forced = 0;
         if (n_forced > d) n_forced = d;
         if (n_free > d - n_forced) n_free = d - n_forced;
         const int total = n_forced + n_free;
-        const bool outliers = quant && (a.flags & OBC_FLAG_OUTLIERS);
+        const bool outliers = Q && quant && (a.flags & OBC_FLAG_OUTLIERS);
 
         // ---- row set-up ------------------------------------------------------------------------------
         for (int j = tid; j < d; j += NT) {
@@ -342,8 +362,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             if (a.mask) a.mask[(size_t)r * d + j] = 1;
         }
         if (has_nm) for (int b = tid; b < (d >> nm_lg); b += NT) blkcnt[b] = 0;
-        for (int j = d + tid; j < cap; j += NT) perm[j] = -1;
         for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
+        for (int j = d + tid; j < cap; j += NT) perm[j] = -1;
         if (tid == 0) {
             bc->sc = 1.0; bc->ze = 0.0; bc->mq = 0.0;
             if (a.mode == MODE_QUANT) {
@@ -437,9 +457,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 }
             }
             const bool forced = s < n_forced;
-            const bool q_now = quant && !forced;
+            const bool q_now = Q && quant && !forced;
             // ---- grid of the compound path: built from the survivors when the replay is over -----------
-            if (a.mode == MODE_REPLAY_QUANT && s == n_forced) {
+            if (Q && a.mode == MODE_REPLAY_QUANT && s == n_forced) {
                 float lo = 0.f, hi = 0.f;
 #pragma unroll
                 for (int k = 0; k < KMAX; ++k) {               // own slots: their owner is the only writer
@@ -475,9 +495,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 }
             } else {
                 if (!sa_valid || tail || outliers)
-                    estimate_own<NT, KMAX>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq, has_nm ? blkcnt : nullptr,
+                    estimate_own<NT, KMAX, Q>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq, has_nm ? blkcnt : nullptr,
                                            nm_lg, nm_prune, cntw);
-                thread_best<NT, KMAX>(sa, wd, dg, perm, q_now, outliers, gsc, gisc, gze, gmq, &key, &cs, &cslot);
+                thread_best<NT, KMAX, Q>(sa, wd, dg, perm, q_now, outliers, gsc, gisc, gze, gmq, &key, &cs, &cslot);
             }
             const Records rec = rec_view(scratch, s & 1);
             const Pick pk = block_pick<NT>(key, cs, cslot, cslot >= 0 ? perm[cslot] : -1,
@@ -486,7 +506,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             const double dpp = pk.dgv, wp = pk.w;
             if (p < 0 || !(dpp > 0.0) || !isfinite(dpp) || !isfinite(wp)) { failed = true; break; }
             double qp = 0.0, code = -1.0;
-            if (q_now) qp = grid_q(wp, gsc, gze, gmq, &code);
+            if (Q && q_now) qp = grid_q(wp, gsc, gze, gmq, &code);
             const double e = wp - qp;
             if (!tail) {
                 // ======================= deferred-update step ==============================================
@@ -537,7 +557,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 // state update of the own slots (Eq. 3 / Eq. 7), the new pending vector, and the score
                 // estimates the next free step starts from
                 const bool est_next = (s + 1 >= n_forced) && !outliers;
-                const bool q_next = quant && (s + 1 >= n_forced);
+                const bool q_next = Q && quant && (s + 1 >= n_forced);
 #pragma unroll
                 for (int g = 0; g < KMAX / 4; ++g) {
                     const int jb = own_slot<NT>(4 * g);
@@ -561,7 +581,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         const double nd = dg[j] - (double)vj * (double)vj * idpp;
                         wd[j] = nw; dg[j] = nd;
                         zv[q] = vj * rs;
-                        if (est_next) sa[k] = score_estimate(nw, nd, q_next, gsc, gisc, gze, gmq);
+                        if (est_next) sa[k] = score_estimate<Q>(nw, nd, q_next, gsc, gisc, gze, gmq);
                         if (has_nm) {
                             if ((pq[q] >> nm_lg) == (op >> nm_lg)) cntw[g] += 1u << (8 * q);
                             if ((int)((cntw[g] >> (8 * q)) & 0xFFu) >= nm_prune) sa[k] = CUDART_NAN_F;
@@ -673,7 +693,7 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false) {
     const int cap = (d + 3) & ~3;
     int nt = engine_threads_choice();
-    if (nt != 128 && nt != 256 && nt != 512) nt = d <= 1024 ? 128 : (d <= 2048 ? 256 : 512);
+    if (nt != 128 && nt != 256 && nt != 512) nt = d <= 512 ? 128 : (d <= 2048 ? 256 : 512);
     if (nt == 128 && cap > 1024) nt = 256;
     if (nt == 256 && cap > 2048) nt = 512;
     BlkPlan p;
@@ -720,15 +740,22 @@ obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
     return OBC_OK;
 }
 
-template <int NT, int KMAX>
-static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <int NT, int KMAX, bool Q>
+static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
+    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
-    blocked_engine_kernel<NT, KMAX><<<blocks, NT, smem, stream>>>(a);
+    blocked_engine_kernel<NT, KMAX, Q><<<blocks, NT, smem, stream>>>(a);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
+
+template <int NT, int KMAX>
+static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
+    const bool q = a.mode == MODE_QUANT || a.mode == MODE_REPLAY_QUANT;
+    return q ? blk_launch_q<NT, KMAX, true>(a, blocks, smem, stream) : blk_launch_q<NT, KMAX, false>(a, blocks, smem, stream);
+}
+static obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream);
 
 obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
     DeviceInfo di;
@@ -751,9 +778,13 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
         if (!ws || !aligned256(ws) || ws_bytes < need) return OBC_ERR_WORKSPACE;
         a.Hws = reinterpret_cast<float*>(ws);
     }
-    if (p.nt == 128) return blk_launch<128, 8>(a, blocks, p.smem, stream);
-    if (p.nt == 256) return blk_launch<256, 8>(a, blocks, p.smem, stream);
-    return blk_launch<512, 12>(a, blocks, p.smem, stream);
+    return blk_launch_nt(a, p.nt, blocks, p.smem, stream);
+}
+
+obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream) {
+    if (nt == 128) return blk_launch<128, 8>(a, blocks, smem, stream);
+    if (nt == 256) return blk_launch<256, 8>(a, blocks, smem, stream);
+    return blk_launch<512, 12>(a, blocks, smem, stream);
 }
 
 }  // namespace obc
