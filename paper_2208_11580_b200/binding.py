@@ -100,7 +100,8 @@ def obc_engine_plan(d_col: int, with_trace: bool = False) -> dict:
     plan = (ctypes.c_int32 * 8)()
     _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), plan), "obc_engine_plan")
     return {"engine": int(plan[0]), "threads": int(plan[1]), "rows_per_sm": int(plan[2]), "on_chip_below": int(plan[3]),
-            "panel_floats": int(plan[4]), "max_pending": int(plan[5]), "sm_count": int(plan[6])}
+            "panel_floats": int(plan[4]), "max_pending": int(plan[5]), "sm_count": int(plan[6]),
+            "l2_vectors": int(plan[7])}
 
 
 def _ptr(t):

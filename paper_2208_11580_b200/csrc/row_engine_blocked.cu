@@ -138,7 +138,10 @@ template <bool Q>
 __device__ __forceinline__ float score_estimate(double w, double dgv, bool quant, double sc, double isc, double ze,
                                                 double mq) {
     if (Q && quant) {
-        const double err = grid_error(w, sc, isc, ze, mq);
+        // plain product and rounding: next to a rounding boundary the two possible codes give the same |err| to
+        // ~1e-16, which is all an estimate needs (the exact scoring goes through grid_error)
+        const double c = fmin(fmax(rint(w * isc) + ze, 0.0), mq);
+        const double err = sc * (c - ze) - w;
         return __fdividef(__double2float_rn(err * err), __double2float_rn(dgv));
     }
     const float wf = __double2float_rn(w);
@@ -218,9 +221,51 @@ __device__ __forceinline__ void thread_best(const float (&sa)[KMAX], const doubl
 // A warp works on tiles of RG rows x 128 columns (row groups dealt out cyclically to the warps); each lane keeps
 // its RG x 4 sub-tile in registers, so RG x 16 bytes per lane are in flight while a tile is fetched and the
 // pending vectors cost RG/4 + 1 shared-memory loads per 4 RG multiply-adds.
-template <int NT, int RG>
-__device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m1, int nb, const float* Z, int ldz,
-                                          const unsigned short* srcm, const uint32_t* colmask) {
+// The first nbs vectors are rows of Z (shared memory, stride ldz), the others rows of G (global memory, stride gld:
+// the overflow part of the pending vectors, small enough to stay in L2).  STREAM: the triangle is far larger than
+// L2 and touched once per flush, so it is loaded and stored with the evict-first hint and leaves L2 to G.
+template <int RG>
+__device__ __forceinline__ void flush_apply_vector(float4 (&acc)[RG], const float* zb, int i0, int j) {
+    const float4 zj = *reinterpret_cast<const float4*>(zb + j);
+#pragma unroll
+    for (int r4 = 0; r4 < RG / 4; ++r4) {
+        const float4 za = *reinterpret_cast<const float4*>(zb + i0 + 4 * r4);
+        const float zi[4] = {za.x, za.y, za.z, za.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float4& t = acc[4 * r4 + q];
+            t.x = fmaf(-zi[q], zj.x, t.x);
+            t.y = fmaf(-zi[q], zj.y, t.y);
+            t.z = fmaf(-zi[q], zj.z, t.z);
+            t.w = fmaf(-zi[q], zj.w, t.w);
+        }
+    }
+}
+
+// Same with the column operand already in registers and the row operand in a small shared-memory block
+// (zrow[0..RG)): used for the overflow vectors, whose column operands are prefetched from L2.
+template <int RG>
+__device__ __forceinline__ void flush_apply_staged(float4 (&acc)[RG], const float4 zj, const float* zrow) {
+#pragma unroll
+    for (int r4 = 0; r4 < RG / 4; ++r4) {
+        const float4 za = *reinterpret_cast<const float4*>(zrow + 4 * r4);
+        const float zi[4] = {za.x, za.y, za.z, za.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float4& t = acc[4 * r4 + q];
+            t.x = fmaf(-zi[q], zj.x, t.x);
+            t.y = fmaf(-zi[q], zj.y, t.y);
+            t.z = fmaf(-zi[q], zj.z, t.z);
+            t.w = fmaf(-zi[q], zj.w, t.w);
+        }
+    }
+}
+
+// zstage: per-warp staging block of (nb - nbs) x RG floats for the row operands of the overflow vectors.
+template <int NT, int RG, bool STREAM>
+__device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m1, int nb, int nbs, const float* Z,
+                                          int ldz, const float* G, int gld, float* zstage, const unsigned short* srcm,
+                                          const uint32_t* colmask) {
     constexpr int NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nrg = (m1 + RG - 1) / RG;
@@ -231,6 +276,16 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 #pragma unroll
         for (int r = 0; r < RG; ++r) sr[r] = (r < nrows) ? (int)srcm[i0 + r] : i0;
         const int jend = i0 + nrows;                           // columns [0, jend) hold data of this row group
+        const int nbg = nb - nbs;
+        if (nbg > 0) {                                         // row operands of the overflow vectors -> staging block
+            __syncwarp();
+            for (int e = lane; e < nbg * (RG / 4); e += 32) {
+                const int v = e / (RG / 4), q = e - v * (RG / 4);
+                *reinterpret_cast<float4*>(zstage + v * RG + 4 * q) =
+                    *reinterpret_cast<const float4*>(G + (size_t)v * gld + i0 + 4 * q);
+            }
+            __syncwarp();
+        }
         for (int c0 = 0; c0 < jend; c0 += 128) {
             const int j = c0 + (lane << 2);
             if (j >= jend) continue;                           // whole float4 above the diagonal of every row
@@ -238,8 +293,10 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 #pragma unroll
             for (int r = 0; r < RG; ++r) {
                 acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (r < nrows && j <= i0 + r)
-                    acc[r] = *reinterpret_cast<const float4*>(Hp + (size_t)sr[r] * ldp + j);
+                if (r < nrows && j <= i0 + r) {
+                    const float4* src = reinterpret_cast<const float4*>(Hp + (size_t)sr[r] * ldp + j);
+                    acc[r] = STREAM ? __ldcs(src) : *src;
+                }
             }
             // columns of this lane that are holes: their data sits in the mover's row
             const uint32_t my4 = (colmask[j >> 5] >> (j & 31)) & 0xFu;
@@ -260,27 +317,26 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
                     }
                 }
             }
-            for (int b = 0; b < nb; ++b) {
-                const float* zb = Z + (size_t)b * ldz;
-                const float4 zj = *reinterpret_cast<const float4*>(zb + j);
-#pragma unroll
-                for (int r4 = 0; r4 < RG / 4; ++r4) {
-                    const float4 za = *reinterpret_cast<const float4*>(zb + i0 + 4 * r4);
-                    const float zi[4] = {za.x, za.y, za.z, za.w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float4& t = acc[4 * r4 + q];
-                        t.x = fmaf(-zi[q], zj.x, t.x);
-                        t.y = fmaf(-zi[q], zj.y, t.y);
-                        t.z = fmaf(-zi[q], zj.z, t.z);
-                        t.w = fmaf(-zi[q], zj.w, t.w);
-                    }
+            for (int b = 0; b < nbs; ++b) flush_apply_vector<RG>(acc, Z + (size_t)b * ldz, i0, j);
+            if (nbg > 0) {                                     // column operands from L2, two vectors ahead
+                const float* gj = G + j;
+                float4 q0 = *reinterpret_cast<const float4*>(gj), q1 = q0;
+                if (nbg > 1) q1 = *reinterpret_cast<const float4*>(gj + gld);
+                for (int b = 0; b < nbg; b += 2) {
+                    float4 n0 = q0, n1 = q1;
+                    if (b + 2 < nbg) n0 = *reinterpret_cast<const float4*>(gj + (size_t)(b + 2) * gld);
+                    if (b + 3 < nbg) n1 = *reinterpret_cast<const float4*>(gj + (size_t)(b + 3) * gld);
+                    flush_apply_staged<RG>(acc, q0, zstage + b * RG);
+                    if (b + 1 < nbg) flush_apply_staged<RG>(acc, q1, zstage + (b + 1) * RG);
+                    q0 = n0; q1 = n1;
                 }
             }
 #pragma unroll
             for (int r = 0; r < RG; ++r)
-                if (r < nrows && j <= i0 + r)
-                    *reinterpret_cast<float4*>(Hp + (size_t)(i0 + r) * ldp + j) = acc[r];
+                if (r < nrows && j <= i0 + r) {
+                    float4* dst = reinterpret_cast<float4*>(Hp + (size_t)(i0 + r) * ldp + j);
+                    if (STREAM) __stcs(dst, acc[r]); else *dst = acc[r];
+                }
         }
     }
 }
@@ -335,6 +391,12 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     const int lds = ms + 1;
     float* Hp = a.Hws ? a.Hws + (size_t)blockIdx.x * d * a.ldp : nullptr;
     const int ldp = a.ldp;
+    // overflow of the pending vectors: gB more of them in global memory (sized to stay in L2), stride gld
+    // (only the one-row-per-SM configuration uses it; the other kernels are built without that code)
+    constexpr bool GP = NT >= 512;
+    const int gB = (GP && a.Gpan) ? a.g_vectors : 0, gld = a.g_ld;
+    float* G = (GP && a.Gpan) ? a.Gpan + (size_t)blockIdx.x * a.g_vectors * a.g_ld : nullptr;
+    float* zstage = panel + a.panel_floats + (size_t)warp * a.g_vectors * 16;    // per warp: g_vectors x 16 floats
 
     for (int rr = blockIdx.x; rr < a.row_count; rr += gridDim.x) {
         const int r = a.row_begin + rr;
@@ -390,7 +452,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         int m0 = d;                      // slots in use (tail phase: number of live slots)
         int nb = 0;                      // pending vectors
         int ldz = (m0 + 15) & ~15;
-        int bcur = min(a.max_pending, a.panel_floats / ldz);
+        int scap = a.panel_floats / ldz;     // pending vectors that fit into shared memory at this row length
+        int bcur = min(a.max_pending, scap + gB);
         int s = 0;
         bool failed = false;
         float sa[KMAX];                  // score estimates of the own slots, kept up to date by the update phase
@@ -420,7 +483,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     const int nh = bc->nh;
                     for (int idx = tid; idx < nh * nb; idx += NT) {
                         const int q = idx / nb, b = idx - q * nb;
-                        panel[(size_t)b * ldz + hl[q]] = panel[(size_t)b * ldz + mv[q]];
+                        float* zr = (!GP || b < scap) ? panel + (size_t)b * ldz : G + (size_t)(b - scap) * gld;
+                        zr[hl[q]] = zr[mv[q]];
                     }
                     if (tid < nh) {
                         const int h = hl[tid];
@@ -428,7 +492,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         atomicOr(&colmask[h >> 5], 1u << (h & 31));
                     }
                     __syncthreads();
-                    blk_flush<NT, 16>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
+                    blk_flush<NT, 16, (NT >= 512)>(Hp, ldp, m1, nb, GP ? min(nb, scap) : nb, panel, ldz, G, gld, zstage, srcm, colmask);
                     __syncthreads();
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
@@ -443,7 +507,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 #pragma unroll
                     for (int g = 0; g < KMAX / 4; ++g) cntw[g] = 0u;
                     ldz = (m0 + 15) & ~15;
-                    bcur = min(a.max_pending, a.panel_floats / ldz);
+                    scap = a.panel_floats / ldz;
+                    bcur = min(a.max_pending, scap + gB);
                     __syncthreads();
                 }
                 if (m0 <= ms) {
@@ -510,7 +575,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             const double e = wp - qp;
             if (!tail) {
                 // ======================= deferred-update step ==============================================
-                float* zb = panel + (size_t)nb * ldz;
+                float* zb = (!GP || nb < scap) ? panel + (size_t)nb * ldz : G + (size_t)(nb - scap) * gld;
                 // pivot column of the stored matrix (own slots), corrected by the pending vectors
                 float c[KMAX], corr[KMAX];
                 unsigned live = 0u;
@@ -540,8 +605,25 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 const double idpp = 1.0 / dpp;
                 const double f = e * idpp;
                 const float rs = __frsqrt_rn((float)dpp);
-                for (int b = 0; b < nb; ++b) {
+                const int nbs = GP ? min(nb, scap) : nb;
+                for (int b = 0; b < nbs; ++b) {
                     const float* zo = panel + (size_t)b * ldz;
+                    const float zp = zo[p];
+#pragma unroll
+                    for (int g = 0; g < KMAX / 4; ++g) {
+                        if ((live >> (4 * g)) & 0xFu) {
+                            const float4 z = *reinterpret_cast<const float4*>(zo + own_slot<NT>(4 * g));
+                            corr[4 * g] = fmaf(z.x, zp, corr[4 * g]);
+                            corr[4 * g + 1] = fmaf(z.y, zp, corr[4 * g + 1]);
+                            corr[4 * g + 2] = fmaf(z.z, zp, corr[4 * g + 2]);
+                            corr[4 * g + 3] = fmaf(z.w, zp, corr[4 * g + 3]);
+                        }
+                    }
+                }
+                if (GP)
+#pragma unroll 2
+                for (int b = nbs; b < nb; ++b) {               // the overflow vectors, from L2
+                    const float* zo = G + (size_t)(b - scap) * gld;
                     const float zp = zo[p];
 #pragma unroll
                     for (int g = 0; g < KMAX / 4; ++g) {
@@ -608,7 +690,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     __syncthreads();
                     for (int j = tid; j < d; j += NT)
                         a.w_trace[((size_t)r * (a.trace_steps + 1) + s + 1) * d + j] = wfull[j];
-                    __syncthreads();                           // wfull is written again in the next step
+                    // wfull is next written in the update phase of the following step, i.e. behind that step's
+                    // barrier, which every thread reaches only after these reads
                 }
             } else {
                 // ======================= on-chip step (compaction at every step) ===========================
@@ -679,7 +762,11 @@ struct BlkPlan {
     size_t smem;       // dynamic shared memory per block
     int panel_floats;
     int ms;
+    int g_vectors;     // overflow pending vectors per block in global memory (0 = none)
+    int g_ld;          // their stride in floats
 };
+
+constexpr size_t BLK_L2_PANEL_BUDGET = (size_t)48 << 20;      // all blocks' overflow vectors together: well inside L2
 
 static int blk_pick_ms(int d, size_t panel_bytes) {
     int ms = d < 1024 ? d : 1024;
@@ -714,6 +801,23 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     p.smem = share;
     p.panel_floats = (int)((share - fixed) / 4);
     p.ms = blk_pick_ms(d, share - fixed);
+    // Very long rows (d_col > ~2600): shared memory holds fewer than 16 pending vectors and the flush is bound by
+    // the traffic of the triangle; further vectors go to a global buffer small enough to stay in L2 (the triangle
+    // itself is streamed past it with evict-first hints).  Measured at d_col = 3072: 99 -> 83 ms per wave of rows;
+    // at 2304 (19 vectors in shared memory) it gains nothing, so it is not used there.
+    p.g_ld = (cap + 15) & ~15;
+    p.g_vectors = 0;
+    if (p.nt == 512) {
+        const int in_smem = p.panel_floats / p.g_ld;
+        int g = (int)(BLK_L2_PANEL_BUDGET / ((size_t)di.sm_count * p.g_ld * 4));
+        if (g > 32) g = 32;
+        const size_t stage = (size_t)(p.nt / 32) * g * 16 * 4;     // per-warp staging of their row operands
+        if (in_smem < 16 && g >= 4 && share - fixed >= stage + 4 * min_panel) {
+            p.g_vectors = g;
+            p.panel_floats = (int)((share - fixed - stage) / 4);
+            p.ms = blk_pick_ms(d, share - fixed - stage);
+        }
+    }
     *out = p;
     return true;
 }
@@ -725,7 +829,9 @@ size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di
     const int cap = (d + 3) & ~3;
     int blocks = di.sm_count * 4;                 // the largest grid any thread-count choice uses
     if (row_count > 0 && row_count < blocks) blocks = row_count;
-    return round_up((size_t)blocks * d * cap * sizeof(float), 256);
+    const int gblocks = blocks < di.sm_count ? blocks : di.sm_count;     // overflow vectors: one block per SM only
+    return round_up((size_t)blocks * d * cap * sizeof(float), 256) +
+           round_up((size_t)gblocks * BLK_MAXB * ((cap + 15) & ~15) * sizeof(float), 256);
 }
 
 obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
@@ -736,7 +842,7 @@ obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
     if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p)) return OBC_ERR_UNSUPPORTED;
     const int mp = engine_pending_choice();
     plan[0] = OBC_ENGINE_BLOCKED; plan[1] = p.nt; plan[2] = p.per_sm; plan[3] = p.ms; plan[4] = p.panel_floats;
-    plan[5] = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB; plan[6] = di.sm_count; plan[7] = 0;
+    plan[5] = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB; plan[6] = di.sm_count; plan[7] = p.g_vectors;
     return OBC_OK;
 }
 
@@ -772,11 +878,19 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     int blocks = di.sm_count * p.per_sm;
     if (a.row_count < blocks) blocks = a.row_count;
     a.Hws = nullptr;
+    a.Gpan = nullptr;
+    a.g_vectors = 0;
+    a.g_ld = p.g_ld;
     a.ldp = a.cap;
     if (a.d > p.ms) {
-        const size_t need = round_up((size_t)blocks * a.d * a.cap * sizeof(float), 256);
-        if (!ws || !aligned256(ws) || ws_bytes < need) return OBC_ERR_WORKSPACE;
+        const size_t tri = round_up((size_t)blocks * a.d * a.cap * sizeof(float), 256);
+        const size_t gpan = p.g_vectors ? round_up((size_t)blocks * p.g_vectors * p.g_ld * sizeof(float), 256) : 0;
+        if (!ws || !aligned256(ws) || ws_bytes < tri + gpan) return OBC_ERR_WORKSPACE;
         a.Hws = reinterpret_cast<float*>(ws);
+        if (p.g_vectors) {
+            a.Gpan = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + tri);
+            a.g_vectors = p.g_vectors;
+        }
     }
     return blk_launch_nt(a, p.nt, blocks, p.smem, stream);
 }
