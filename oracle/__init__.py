@@ -128,6 +128,41 @@ def run_rows(Hinv, W, steps=None, mode="prune", scale=None, zero=None, maxq=0, f
     return out
 
 
+def run_rows_blocks(Hinv, W, c: int, steps=None, forced_blocks=None, return_hi=False):
+    """Block pruning (Section 3, "Block-Sparsity", Eq. 5) of every row of W: blocks of c consecutive weights are
+    removed together, chosen by w_P^T ((Hinv)_P)^-1 w_P.  steps = number of blocks to remove (default all).
+    Returns a dict: order, loss (rows x steps*c; a block's loss sits at its first member, zeros after it), margin,
+    best_block, forced_gap (rows x steps), w (rows x d), status (rows), and Hi (list of matrices) if return_hi."""
+    Hinv = np.ascontiguousarray(Hinv, dtype=np.float64)
+    Wd = np.array(W, dtype=np.float64, order="C", copy=True)
+    if Wd.ndim == 1:
+        Wd = Wd[None, :]
+    rows, d = Wd.shape
+    assert 1 <= c <= 8 and d % c == 0
+    steps = d // c if steps is None else int(steps)
+    fo = None if forced_blocks is None else np.ascontiguousarray(np.asarray(forced_blocks, np.int32).reshape(rows, steps))
+    out = dict(order=np.full((rows, steps * c), -1, np.int32), loss=np.zeros((rows, steps * c)),
+               margin=np.ones((rows, steps)), best_block=np.full((rows, steps), -1, np.int32),
+               forced_gap=np.zeros((rows, steps)), status=np.zeros(rows, np.int32))
+    lib = _L()
+    lib.oracle_row_blocks.restype = ctypes.c_int
+    I32, F64 = ctypes.c_int32, ctypes.c_double
+    his = []
+    for r in range(rows):
+        Hi = Hinv.copy()
+        out["status"][r] = lib.oracle_row_blocks(_p(Hi, F64), ctypes.c_int(d), _p(Wd[r], F64), ctypes.c_int(c),
+                                                 ctypes.c_int(steps), None if fo is None else _p(fo[r], I32),
+                                                 _p(out["order"][r], I32), _p(out["loss"][r], F64),
+                                                 _p(out["margin"][r], F64), _p(out["best_block"][r], I32),
+                                                 _p(out["forced_gap"][r], F64))
+        if return_hi:
+            his.append(Hi)
+    out["w"] = Wd
+    if return_hi:
+        out["Hi"] = his
+    return out
+
+
 def eliminate_one_row(Hinv, w, **kw):
     """Single-row variant that also returns the row's private Hinv copy after the steps ('Hi')."""
     Hi = np.array(Hinv, dtype=np.float64, order="C", copy=True)

@@ -217,6 +217,108 @@ int oracle_row(double *Hi, int d, double *w, int steps, int mode,
     return ret;
 }
 
+/* ---- Block pruning (Section 3, "Block-Sparsity", Eq. 5) ------------------------------------------------------
+ * Zeros appear in blocks of c consecutive weights.  Per step, over the remaining blocks P:
+ *      P*  = argmin_P  w_P^T ((Hinv)_P)^-1 w_P                       (ties: lowest block)
+ *      w  -= Hinv[:,P*] ((Hinv)_P*)^-1 w_P*                          (then w_P* = 0 exactly)
+ *      Hinv: Lemma 1 applied successively for every p in P* (ascending), rows/columns of P* zeroed.
+ * The c x c systems are solved directly by Gaussian elimination with partial pivoting.
+ * order[c*t .. c*t+c) = the members of the t-th block (ascending), loss[c*t] = its score w_P^T((Hinv)_P)^-1 w_P and
+ * loss[c*t+1 .. c*t+c) = 0, so that the per-weight global step (Algorithm 2) takes a block's members together.
+ * forced_blocks (nullable): block index to take at step t instead of the argmin; best_block/forced_gap/margin describe
+ * the oracle's own choice as in oracle_row.  Returns 0, or 1+t when a block matrix is not positive definite. */
+static int solve_small(int c, const double *A, const double *b, double *x)
+{
+    double M[8][9];
+    for (int i = 0; i < c; ++i) { for (int j = 0; j < c; ++j) M[i][j] = A[i * c + j]; M[i][c] = b[i]; }
+    for (int k = 0; k < c; ++k) {
+        int piv = k;
+        for (int i = k + 1; i < c; ++i) if (fabs(M[i][k]) > fabs(M[piv][k])) piv = i;
+        if (!(fabs(M[piv][k]) > 0.0) || !isfinite(M[piv][k])) return 1;
+        if (piv != k) for (int j = 0; j <= c; ++j) { double t = M[k][j]; M[k][j] = M[piv][j]; M[piv][j] = t; }
+        for (int i = k + 1; i < c; ++i) {
+            const double f = M[i][k] / M[k][k];
+            for (int j = k; j <= c; ++j) M[i][j] -= f * M[k][j];
+        }
+    }
+    for (int i = c - 1; i >= 0; --i) {
+        double t = M[i][c];
+        for (int j = i + 1; j < c; ++j) t -= M[i][j] * x[j];
+        x[i] = t / M[i][i];
+    }
+    return 0;
+}
+
+int oracle_row_blocks(double *Hi, int d, double *w, int c, int steps, const int32_t *forced_blocks,
+                      int32_t *order, double *loss, double *margin, int32_t *best_block, double *forced_gap)
+{
+    const double tiny = 1e-300;
+    const int nblk = d / c;
+    uint8_t *gone = (uint8_t *)calloc((size_t)nblk, 1);
+    double A[64], x[8], wp[8];
+    int ret = 0;
+    for (int t = 0; t < steps; ++t) {
+        int b = -1, b2 = -1;
+        double sb = 0.0, sb2 = 0.0, sforced = 0.0;
+        const int fb = forced_blocks ? forced_blocks[t] : -1;
+        for (int q = 0; q < nblk; ++q) {
+            if (gone[q]) continue;
+            for (int i = 0; i < c; ++i) {
+                wp[i] = w[q * c + i];
+                for (int j = 0; j < c; ++j) A[i * c + j] = Hi[(int64_t)(q * c + i) * d + q * c + j];
+            }
+            if (solve_small(c, A, wp, x)) { ret = ret ? ret : 1 + t; break; }
+            double s = 0.0;
+            for (int i = 0; i < c; ++i) s += wp[i] * x[i];
+            if (!(s >= 0.0) || !isfinite(s)) { ret = ret ? ret : 1 + t; break; }
+            if (q == fb) sforced = s;
+            if (b < 0 || s < sb) { b2 = b; sb2 = sb; b = q; sb = s; }
+            else if (b2 < 0 || s < sb2) { b2 = q; sb2 = s; }
+        }
+        if (ret || b < 0) { ret = ret ? ret : 1 + t; break; }
+        int P = b;
+        double sp = sb;
+        if (forced_blocks) {
+            if (fb < 0 || fb >= nblk || gone[fb]) { ret = 1 + t; break; }
+            P = fb; sp = sforced;
+        }
+        if (best_block) best_block[t] = b;
+        if (margin) margin[t] = (b2 < 0) ? 1.0 : (sb2 - sb) / fmax(sb2, tiny);
+        if (forced_gap) forced_gap[t] = (sp - sb) / fmax(sp, tiny);
+        for (int i = 0; i < c; ++i) { order[t * c + i] = P * c + i; loss[t * c + i] = 0.0; }
+        loss[t * c] = sp;
+        /* weight update with the block formula (Eq. 5) */
+        for (int i = 0; i < c; ++i) {
+            wp[i] = w[P * c + i];
+            for (int j = 0; j < c; ++j) A[i * c + j] = Hi[(int64_t)(P * c + i) * d + P * c + j];
+        }
+        if (solve_small(c, A, wp, x)) { ret = 1 + t; break; }
+        for (int j = 0; j < d; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < c; ++i) acc += Hi[(int64_t)j * d + P * c + i] * x[i];
+            w[j] -= acc;
+        }
+        for (int i = 0; i < c; ++i) w[P * c + i] = 0.0;
+        /* Lemma 1, successively for every member of the block */
+        for (int i = 0; i < c; ++i) {
+            const int p = P * c + i;
+            const double dpp = Hi[(int64_t)p * d + p];
+            if (!(dpp > 0.0) || !isfinite(dpp)) { ret = 1 + t; break; }
+            for (int a = 0; a < d; ++a) {
+                if (a == p) continue;
+                const double g = Hi[(int64_t)a * d + p] / dpp;
+                if (g == 0.0) continue;
+                for (int e = 0; e < d; ++e) Hi[(int64_t)a * d + e] -= g * Hi[(int64_t)p * d + e];
+            }
+            for (int a = 0; a < d; ++a) { Hi[(int64_t)p * d + a] = 0.0; Hi[(int64_t)a * d + p] = 0.0; }
+        }
+        if (ret) break;
+        gone[P] = 1;
+    }
+    free(gone);
+    return ret;
+}
+
 /* Many independent rows (Section 3: no Hessian interaction between rows); OpenMP over rows.
  * Per-row arrays are strided by `steps` (order, loss, margin, best, forced_gap, round_dist, pivot_diag),
  * by d (w, codes, active0) and by (steps+1)*d (w_trace).  scale/zero are per row.  Each row works on

@@ -358,3 +358,51 @@ def test_pin_nm_pattern(nm):
             want |= set(idx.tolist())
         assert set(ro["order"][r].tolist()) == want
         assert np.array_equal(ro["order"][r], np.array(sorted(want, key=lambda j: (score[r, j], j))))
+
+
+@pytest.mark.parametrize("c", [2, 4])
+def test_pin_block_pruning(c):
+    """Block pruning (Section 3, "Block-Sparsity", Eq. 5): (1) every pick is the brute-force minimiser over the remaining
+    blocks of the true loss increase, which is half the recorded block score; (2) after every block step the
+    remaining weights are the masked least-squares optimum and the reduced inverse is inv(H[M,M]); (3) with c = 1 the
+    procedure is Algorithm 1; (4) with a diagonal Hessian the block score is sum w_j^2 H_jj over the block."""
+    d = 12
+    W, X, Hd, Hinv, X_aug = _problem(3, d, 70, 41 + c)
+    nblk = d // c
+    for r in range(W.shape[0]):
+        removed = []
+        for t in range(nblk):
+            res = oracle.run_rows_blocks(Hinv, W[r], c, steps=t + 1, return_hi=True)
+            assert res["status"][0] == 0
+            keep_before = [j for j in range(d) if j not in removed]
+            base = np.sum(((W[r] - _masked_lstsq(W[r], X_aug, keep_before)) @ X_aug) ** 2)
+            inc = {}
+            for q in range(nblk):
+                blk = list(range(q * c, q * c + c))
+                if blk[0] in removed:
+                    continue
+                F = [j for j in keep_before if j not in blk]
+                inc[q] = np.sum(((W[r] - _masked_lstsq(W[r], X_aug, F)) @ X_aug) ** 2) - base
+            best = min(inc, key=lambda q: (inc[q], q))
+            picked = res["order"][0, t * c:(t + 1) * c]
+            assert picked.tolist() == list(range(best * c, best * c + c))
+            assert np.isclose(0.5 * res["loss"][0, t * c], inc[best], rtol=1e-6, atol=1e-12)
+            assert np.all(res["loss"][0, t * c + 1:(t + 1) * c] == 0.0)
+            removed += picked.tolist()
+            keep = [j for j in range(d) if j not in removed]
+            assert np.allclose(res["w"][0], _masked_lstsq(W[r], X_aug, keep), rtol=1e-8, atol=1e-11)
+            assert np.all(res["w"][0][removed] == 0.0)
+            if keep:
+                assert np.allclose(res["Hi"][0][np.ix_(keep, keep)], np.linalg.inv(Hd[np.ix_(keep, keep)]), rtol=1e-8, atol=1e-13)
+    one = oracle.run_rows_blocks(Hinv, W, 1)
+    ref = oracle.run_rows(Hinv, W)
+    assert np.array_equal(one["order"], ref["order"]) and np.allclose(one["loss"], ref["loss"], rtol=1e-12)
+    assert np.allclose(one["w"], ref["w"], atol=1e-14)
+    Wo, Xo = obc_synth.make_small(2, d, 40, 5, "orthogonal")
+    Ho = np.diag(np.diag(oracle.hessian(Xo, True)))
+    Hio, _ = oracle.inverse(Ho, 0.0)
+    ro = oracle.run_rows_blocks(Hio, Wo, c)
+    score = (Wo.astype(np.float64) ** 2 * np.diag(Ho)).reshape(2, nblk, c).sum(axis=2)
+    for r in range(2):
+        assert np.array_equal(ro["order"][r, ::c] // c, np.argsort(score[r], kind="stable"))
+        assert np.allclose(ro["loss"][r, ::c], np.sort(score[r]), rtol=1e-12)
