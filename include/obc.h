@@ -57,7 +57,7 @@ enum {
 
 typedef enum {
     OBC_OP_HESSIAN = 0, OBC_OP_INVERSE = 1, OBC_OP_PRUNE_TRACE = 2, OBC_OP_SELECT = 3,
-    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5
+    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5, OBC_OP_PRUNE_BLOCKS = 6
 } obc_op;
 
 /* Which row elimination engine obc_prune_trace / obc_prune_apply / obc_quantize run (all compute Algorithm 1 /
@@ -145,6 +145,21 @@ obc_status obc_prune_nm(const float *W, int ldw, int d_row, int d_col, int row_b
                         const float *Hinv, int ldhi, int n_keep, int m_block,
                         int32_t *order, float *loss, float *W_out, int ldwo, uint8_t *mask, int32_t *row_status,
                         void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Section 3, "Block-Sparsity" (Eq. 5): Algorithm 1 on blocks of `block` consecutive columns.  Each step removes the
+ * remaining block P with the smallest w_P^T ((Hinv)_P)^-1 w_P (ties: lowest block), compensates the other weights by
+ * -Hinv[:,P] ((Hinv)_P)^-1 w_P and eliminates the members of P from the row's inverse Hessian one after the other
+ * (Lemma 1) -- which is the same as eliminating the members singly in ascending order, and that is how it runs.
+ *   block = 4 (the only size built); d_col a multiple of 4.  Full trace (all d_col / 4 blocks).
+ *   order : d_row x d_col, the members of the t-th block at [4t, 4t+4), ascending.
+ *   loss  : d_row x d_col, loss[r][4t] = the block's score, loss[r][4t+1..4t+3] = 0, so that
+ *           obc_select_global_mask with k a multiple of 4 takes whole blocks, and obc_prune_apply works unchanged.
+ *   w_trace: as in obc_prune_trace (one row per single elimination), nullable.
+ * Always runs on the BLOCKED engine.  Workspace: obc_workspace_bytes(OBC_OP_PRUNE_BLOCKS, row_count, d_col, 0). */
+obc_status obc_prune_blocks(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                            const float *Hinv, int ldhi, int block,
+                            int32_t *order, float *loss, float *w_trace, int32_t *row_status,
+                            void *ws, size_t ws_bytes, obc_stream stream);
 
 /* Algorithm 2 (appendix, "ExactOBS Global Step"): repeatedly prune, across all rows, the weight whose
  * next recorded loss is smallest (ties: lowest row), k times.  k is a count, 0 <= k <= d_row*d_col.

@@ -13,13 +13,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIBPATH = os.path.join(_HERE, "libobc.so")
 
-OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE = range(6)
+OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS = range(7)
 PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
 FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm",
+    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -66,6 +66,8 @@ def load_library():
     lib.obc_prune_nm.restype = c_int
     lib.obc_prune_nm.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, c_int, vp, vp, vp, c_int, vp, vp,
                                  vp, c_sz, vp]
+    lib.obc_prune_blocks.restype = c_int
+    lib.obc_prune_blocks.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
     lib.obc_select_global_mask.restype = c_int
     lib.obc_select_global_mask.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp, c_sz, vp]
     lib.obc_select_global_mask_static.restype = c_int
@@ -196,6 +198,19 @@ def obc_prune_nm(W, Hinv, n_keep, m_block, W_out, row_status, order=None, loss=N
     _raise(load_library().obc_prune_nm(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), int(n_keep),
                                        int(m_block), _ptr(order), _ptr(loss), _ptr(W_out), _ld(W_out), _ptr(mask),
                                        _ptr(row_status), _ptr(ws), nb, _stream(stream)), "obc_prune_nm")
+
+
+def obc_prune_blocks(W, Hinv, order, loss, row_status, block=4, w_trace=None, row_begin=0, row_count=None, ws=None,
+                     stream=None):
+    """Block pruning (blocks of `block` consecutive columns, Eq. 5) of rows [row_begin, row_begin+row_count): full trace."""
+    _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(order, torch.int32, "order")
+    _check(loss, torch.float32, "loss"); _check(row_status, torch.int32, "row_status"); _check(w_trace, torch.float32, "w_trace")
+    R, d = W.shape
+    row_count = R - row_begin if row_count is None else row_count
+    ws, nb = _workspace(ws, OP_PRUNE_BLOCKS, row_count, d, 0, W.device, "obc_prune_blocks")
+    _raise(load_library().obc_prune_blocks(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), int(block),
+                                           _ptr(order), _ptr(loss), _ptr(w_trace), _ptr(row_status), _ptr(ws), nb,
+                                           _stream(stream)), "obc_prune_blocks")
 
 
 def obc_select_global_mask(loss, order, k, counts, mask, ws=None, stream=None):

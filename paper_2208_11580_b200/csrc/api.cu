@@ -87,6 +87,11 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
         case OBC_OP_HESSIAN: return n > 0 ? hessian_workspace_bytes(d_col, n) : 0;
         case OBC_OP_INVERSE: return inverse_workspace_bytes(d_col);
         case OBC_OP_SELECT: return row_count > 0 ? select_workspace_bytes(row_count, d_col) : 0;
+        case OBC_OP_PRUNE_BLOCKS: {
+            DeviceInfo di;
+            if (device_info(&di) != OBC_OK || d_col > OBC_MAX_DCOL) return 0;
+            return engine_blocks_workspace_bytes(row_count, d_col, di);
+        }
         case OBC_OP_PRUNE_TRACE:
         case OBC_OP_PRUNE_APPLY:
         case OBC_OP_QUANTIZE: {
@@ -143,6 +148,18 @@ obc_status obc_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_b
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_prune_nm(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, n_keep, m_block, order, loss, W_out,
                            ldwo, mask, row_status, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+obc_status obc_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                            const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
+                            int32_t* row_status, void* ws, size_t ws_bytes, obc_stream stream) {
+    if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (!order || !loss || !row_status || d_col % 4 != 0) return OBC_ERR_INVALID_ARG;
+    if (block != 4 || d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    return engine_prune_blocks(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, block, order, loss, w_trace,
+                               row_status, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 obc_status obc_select_global_mask(const float* loss, const int32_t* order, int d_row, int d_col, int64_t k,

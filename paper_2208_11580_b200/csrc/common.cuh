@@ -80,6 +80,10 @@ obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int ro
                            const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
                            float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
                            cudaStream_t stream);
+obc_status engine_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                               const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
+                               int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream);
+size_t engine_blocks_workspace_bytes(int row_count, int d, const DeviceInfo& di);
 obc_status engine_replay(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                          const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts, float* W_out,
                          int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream);

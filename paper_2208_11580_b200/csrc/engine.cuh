@@ -29,6 +29,7 @@ struct EngineArgs {
     int nm_prune; int nm_lg;              // blocked engine, N:M pattern: at most nm_prune eliminations per block of
                                           // 2^nm_lg consecutive columns (nm_prune = 0: no pattern)
     uint8_t* mask;                        // blocked engine, nullable: d_row x d mask, 0 at eliminated columns
+    int block_c;                          // blocked engine: 4 = block pruning in blocks of 4 columns (Eq. 5), 0 = off
     float* Gpan; int g_vectors; int g_ld; // blocked engine: overflow pending vectors in global memory (per block
                                           // g_vectors rows of g_ld floats), nullptr = none
 };

@@ -458,6 +458,27 @@ obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int ro
     return blocked_engine_launch(a, ws, ws_bytes, stream);      // the pattern is built into the blocked engine only
 }
 
+obc_status engine_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
+                               const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
+                               int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    (void)d_row;
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    a.mode = MODE_PRUNE; a.steps = d_col; a.order = order; a.loss = loss; a.w_trace = w_trace; a.trace_steps = d_col;
+    a.block_c = block;
+    return blocked_engine_launch(a, ws, ws_bytes, stream);
+}
+
+// Block pruning keeps every row in global memory to the end (no on-chip tail), so it needs the private triangles
+// at any row length.
+size_t engine_blocks_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
+    const int cap = (d + 3) & ~3;
+    int blocks = di.sm_count * 4;
+    if (row_count > 0 && row_count < blocks) blocks = row_count;
+    const size_t tri = round_up((size_t)blocks * d * cap * sizeof(float), 256);
+    const size_t other = blocked_engine_workspace_bytes(row_count, d, di);
+    return tri > other ? tri + 256 : other;
+}
+
 obc_status engine_replay(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                          const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts, float* W_out,
                          int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {

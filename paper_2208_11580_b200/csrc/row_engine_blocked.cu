@@ -42,9 +42,10 @@ constexpr int BLK_FIXED = 3200;
 
 // Per-row state in shared memory: wd, dg (FP64), perm (int32), srcm (uint16); optional: the row in original
 // order (weight trace), one byte per block of the N:M pattern.
-__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm = false) {
+// (block pruning: the 6 off-diagonal entries of every 4-slot group's 4 x 4 diagonal block, FP64)
+__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm = false, bool bc = false) {
     return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0) +
-           (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0);
+           (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0) + (bc ? (size_t)12 * cap : 0);
 }
 static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
 
@@ -70,7 +71,7 @@ __device__ __forceinline__ unsigned float_key(float x) {
 }
 constexpr unsigned KEY_NONE = 0xFFFFFFFFu;
 
-struct Pick { int slot; int orig; double w; double dgv; };
+struct Pick { int slot; int orig; double w; double dgv; double s; };
 
 // Combines one candidate per lane into the lane holding the smallest (s, orig); key = float_key((float)s)
 // orders all but near-equal candidates, which are then compared exactly.  Returns the winning lane or -1.
@@ -113,8 +114,8 @@ __device__ __forceinline__ Pick block_pick(unsigned key, double s, int slot, int
     const int o2 = (in && k2 != KEY_NONE) ? rec.orig[lane] : 0x7fffffff;
     const int ww = warp_winner(k2, s2, o2);
     Pick p;
-    p.slot = -1; p.orig = -1; p.w = 0.0; p.dgv = 0.0;
-    if (ww >= 0) { p.slot = rec.slot[ww]; p.orig = rec.orig[ww]; p.w = rec.w[ww]; p.dgv = rec.dgv[ww]; }
+    p.slot = -1; p.orig = -1; p.w = 0.0; p.dgv = 0.0; p.s = 0.0;
+    if (ww >= 0) { p.slot = rec.slot[ww]; p.orig = rec.orig[ww]; p.w = rec.w[ww]; p.dgv = rec.dgv[ww]; p.s = rec.s[ww]; }
     return p;
 }
 
@@ -358,11 +359,35 @@ __device__ __forceinline__ void blk_pass_shared(float* S, int lds, int mp, int p
     }
 }
 
+// Block pruning (Section 3, "Block-Sparsity", Eq. 5), blocks of 4: score w_P^T ((Hinv)_P)^-1 w_P of one 4-slot group
+// from its weights w, the diagonal a_ii and the off-diagonals o = (a01, a02, a03, a12, a13, a23) of its 4 x 4 block, by
+// an LDL^T factorisation: the score is sum_i y_i^2 / d_i, which is also the sum of the four single-weight losses
+// when the members are eliminated in this order.  Returns NaN if the block is not positive definite.
+__device__ __forceinline__ double block4_score(const double* w, const double* a, const double* o) {
+    const double d0 = a[0], r0 = 1.0 / d0;
+    const double l10 = o[0] * r0, l20 = o[1] * r0, l30 = o[2] * r0;
+    const double d1 = a[1] - l10 * o[0], r1 = 1.0 / d1;
+    const double t21 = o[3] - l20 * o[0], t31 = o[4] - l30 * o[0];
+    const double l21 = t21 * r1, l31 = t31 * r1;
+    const double d2 = a[2] - l20 * o[1] - l21 * t21, r2 = 1.0 / d2;
+    const double t32 = o[5] - l30 * o[1] - l31 * t21;
+    const double l32 = t32 * r2;
+    const double d3 = a[3] - l30 * o[2] - l31 * t31 - l32 * t32, r3 = 1.0 / d3;
+    const double y0 = w[0];
+    const double y1 = w[1] - l10 * y0;
+    const double y2 = w[2] - l20 * y0 - l21 * y1;
+    const double y3 = w[3] - l30 * y0 - l31 * y1 - l32 * y2;
+    if (!(d0 > 0.0) || !(d1 > 0.0) || !(d2 > 0.0) || !(d3 > 0.0)) return CUDART_NAN;
+    return y0 * y0 * r0 + y1 * y1 * r1 + y2 * y2 * r2 + y3 * y3 * r3;
+}
+
 // Q = the kernel contains the OBQ code (modes QUANT and REPLAY_QUANT); the pruning kernels are built without it.
-template <int NT, int KMAX, bool Q>
+// BC = 4: block pruning in blocks of 4 consecutive columns (pruning kernels only), 0: single weights.
+template <int NT, int KMAX, bool Q, int BC>
 __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
     extern __shared__ __align__(16) char smem[];
     constexpr int NW = NT / 32;
+    constexpr int BCD = BC ? BC : 1;                           // divisor that is never zero
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int d = a.d, cap = a.cap, ms = a.ms;
     char* scratch = smem;
@@ -381,7 +406,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     const bool has_nm = a.nm_prune > 0;                         // N:M pattern: at most nm_prune eliminations per block
     const int nm_lg = a.nm_lg, nm_prune = a.nm_prune;
     unsigned char* blkcnt = reinterpret_cast<unsigned char*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull));
-    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm));
+    double* boff = reinterpret_cast<double*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm));
+    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm, BC != 0));
     // tail views (step-by-step phase in shared memory) share the panel's space
     const int msr = (ms + 3) & ~3;
     float* tv = panel;
@@ -424,6 +450,13 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             if (a.mask) a.mask[(size_t)r * d + j] = 1;
         }
         if (has_nm) for (int b = tid; b < (d >> nm_lg); b += NT) blkcnt[b] = 0;
+        if (BC) {
+            for (int e = tid; e < (d >> 2) * 6; e += NT) {
+                const int g = e / 6, k = e - g * 6;
+                const int ia = k < 3 ? 0 : (k < 5 ? 1 : 2), ib = k < 3 ? k + 1 : (k < 5 ? k - 1 : 3);
+                boff[e] = (double)a.Hinv[(size_t)(4 * g + ia) * a.ldhi + 4 * g + ib];
+            }
+        }
         for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
         for (int j = d + tid; j < cap; j += NT) perm[j] = -1;
         if (tid == 0) {
@@ -454,8 +487,11 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         int ldz = (m0 + 15) & ~15;
         int scap = a.panel_floats / ldz;     // pending vectors that fit into shared memory at this row length
         int bcur = min(a.max_pending, scap + gB);
+        if (BC) bcur &= ~(BC - 1);           // whole blocks between two flushes, so that 4-slot groups stay together
         int s = 0;
         bool failed = false;
+        int blk_base = 0;                // block pruning: first slot and score of the block being eliminated
+        double blk_score = 0.0;
         float sa[KMAX];                  // score estimates of the own slots, kept up to date by the update phase
         unsigned cntw[KMAX / 4];         // N:M: eliminations so far in the block of each own slot (one byte per slot)
 #pragma unroll
@@ -497,6 +533,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
                         wd[h] = wd[sv]; dg[h] = dg[sv]; perm[h] = perm[sv];
+                        if (BC && (h & 3) == 0)      // holes and movers are whole aligned groups in block mode
+                            for (int k = 0; k < 6; ++k) boff[(h >> 2) * 6 + k] = boff[(sv >> 2) * 6 + k];
                         srcm[h] = (unsigned short)h;
                         colmask[h >> 5] = 0u;
                     }
@@ -509,6 +547,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     ldz = (m0 + 15) & ~15;
                     scap = a.panel_floats / ldz;
                     bcur = min(a.max_pending, scap + gB);
+                    if (BC) bcur &= ~(BC - 1);
                     __syncthreads();
                 }
                 if (m0 <= ms) {
@@ -558,6 +597,25 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     const int j = own_slot<NT>(k);
                     if (j < m0 && perm[j] == f) { cslot = j; key = 0x80000000u; }
                 }
+            } else if (BC && (s - n_forced) % BCD != 0) {
+                // the next member of the block chosen at the last block boundary
+                const int j = blk_base + (s - n_forced) % BCD;
+                if (j >= (tid << 2) && ((j - (tid << 2)) % (4 * NT)) < 4) { cslot = j; key = 0x80000000u; }
+            } else if (BC) {
+                // block boundary: exact FP64 score of every own live group (its four slots are all live here)
+                double bs = CUDART_INF;
+                int bo = 0x7fffffff;
+#pragma unroll
+                for (int g = 0; g < KMAX / 4; ++g) {
+                    const int jb = own_slot<NT>(4 * g);
+                    if (jb < m0 && perm[jb] >= 0) {
+                        const double sc4 = block4_score(wd + jb, dg + jb, boff + (jb >> 2) * 6);
+                        const int o = perm[jb];
+                        if (key_less(sc4, o, bs, bo)) { bs = sc4; bo = o; cslot = jb; }
+                    }
+                }
+                cs = bs;
+                if (cslot >= 0) key = float_key(__double2float_rn(bs));
             } else {
                 if (!sa_valid || tail || outliers)
                     estimate_own<NT, KMAX, Q>(sa, wd, dg, perm, m0, q_now, gsc, gisc, gze, gmq, has_nm ? blkcnt : nullptr,
@@ -569,6 +627,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                                            cslot >= 0 ? wd[cslot] : 0.0, cslot >= 0 ? dg[cslot] : 0.0, rec);
             const int p = pk.slot, op = pk.orig;
             const double dpp = pk.dgv, wp = pk.w;
+            if (BC && !forced && (s - n_forced) % BCD == 0) { blk_base = p; blk_score = pk.s; }
             if (p < 0 || !(dpp > 0.0) || !isfinite(dpp) || !isfinite(wp)) { failed = true; break; }
             double qp = 0.0, code = -1.0;
             if (Q && q_now) qp = grid_q(wp, gsc, gze, gmq, &code);
@@ -638,7 +697,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 }
                 // state update of the own slots (Eq. 3 / Eq. 7), the new pending vector, and the score
                 // estimates the next free step starts from
-                const bool est_next = (s + 1 >= n_forced) && !outliers;
+                const bool est_next = !BC && (s + 1 >= n_forced) && !outliers;
                 const bool q_next = Q && quant && (s + 1 >= n_forced);
 #pragma unroll
                 for (int g = 0; g < KMAX / 4; ++g) {
@@ -671,6 +730,14 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         if (has_wfull) wfull[pq[q]] = (float)nw;
                     }
                     *reinterpret_cast<float4*>(zb + jb) = make_float4(zv[0], zv[1], zv[2], zv[3]);
+                    if (BC && ((live >> (4 * g)) & 0xFu) == 0xFu && jb != (p & ~3)) {
+                        // Lemma 1 on the group's own 4 x 4 diagonal block (off-diagonal part; dg holds the diagonal)
+                        double* o = boff + (jb >> 2) * 6;
+                        const double v0 = (double)(c[4 * g] - corr[4 * g]), v1 = (double)(c[4 * g + 1] - corr[4 * g + 1]);
+                        const double v2 = (double)(c[4 * g + 2] - corr[4 * g + 2]), v3 = (double)(c[4 * g + 3] - corr[4 * g + 3]);
+                        o[0] -= v0 * v1 * idpp; o[1] -= v0 * v2 * idpp; o[2] -= v0 * v3 * idpp;
+                        o[3] -= v1 * v2 * idpp; o[4] -= v1 * v3 * idpp; o[5] -= v2 * v3 * idpp;
+                    }
                 }
                 sa_valid = est_next;
                 if (tid == 0) {
@@ -681,7 +748,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     if (!forced) {
                         const int t = s - n_forced;
                         if (a.order) a.order[(size_t)r * d + t] = op;
-                        if (a.loss) a.loss[(size_t)r * d + t] = (float)(e * e / dpp);
+                        if (a.loss) a.loss[(size_t)r * d + t] = BC ? ((t % BCD) ? 0.f : (float)blk_score) : (float)(e * e / dpp);
                     }
                     if (q_now && a.codes) a.codes[(size_t)r * d + op] = (int)code;
                 }
@@ -777,7 +844,7 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 
 // Threads per block and blocks per SM by row length: short rows are bound by the latency of a step, so
 // several of them share an SM; long rows need the shared memory for pending vectors.
-static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false) {
+static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, bool bc = false) {
     const int cap = (d + 3) & ~3;
     int nt = engine_threads_choice();
     if (nt != 128 && nt != 256 && nt != 512) nt = d <= 512 ? 128 : (d <= 2048 ? 256 : 512);
@@ -790,7 +857,7 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     const size_t sm_total = (size_t)di.smem_optin + 1024;
     size_t share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
     if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
-    const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull, nm);
+    const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull, nm, bc);
     const size_t min_panel = (size_t)4 * ((cap + 15) & ~15);
     while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
         p.per_sm >>= 1;
@@ -846,11 +913,11 @@ obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
     return OBC_OK;
 }
 
-template <int NT, int KMAX, bool Q>
+template <int NT, int KMAX, bool Q, int BC>
 static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
-    blocked_engine_kernel<NT, KMAX, Q><<<blocks, NT, smem, stream>>>(a);
+    blocked_engine_kernel<NT, KMAX, Q, BC><<<blocks, NT, smem, stream>>>(a);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
@@ -859,7 +926,8 @@ static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cud
 template <int NT, int KMAX>
 static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
     const bool q = a.mode == MODE_QUANT || a.mode == MODE_REPLAY_QUANT;
-    return q ? blk_launch_q<NT, KMAX, true>(a, blocks, smem, stream) : blk_launch_q<NT, KMAX, false>(a, blocks, smem, stream);
+    if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4>(a, blocks, smem, stream);
+    return q ? blk_launch_q<NT, KMAX, true, 0>(a, blocks, smem, stream) : blk_launch_q<NT, KMAX, false, 0>(a, blocks, smem, stream);
 }
 static obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream);
 
@@ -870,11 +938,18 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     a.cap = (a.d + 3) & ~3;
     if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     BlkPlan p;
-    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0)) return OBC_ERR_UNSUPPORTED;
+    const bool bc = a.block_c == 4;
+    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc)) return OBC_ERR_UNSUPPORTED;
     a.ms = p.ms;
     a.panel_floats = p.panel_floats;
     int mp = engine_pending_choice();
     a.max_pending = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB;
+    if (bc) {
+        // groups of 4 slots must stay together: no on-chip tail (it compacts slot by slot), whole blocks per flush
+        a.ms = 0;
+        if (a.max_pending < 4) a.max_pending = 4;
+        if (p.panel_floats / p.g_ld + p.g_vectors < 4) return OBC_ERR_UNSUPPORTED;
+    }
     int blocks = di.sm_count * p.per_sm;
     if (a.row_count < blocks) blocks = a.row_count;
     a.Hws = nullptr;
@@ -882,7 +957,7 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     a.g_vectors = 0;
     a.g_ld = p.g_ld;
     a.ldp = a.cap;
-    if (a.d > p.ms) {
+    if (a.d > a.ms) {
         const size_t tri = round_up((size_t)blocks * a.d * a.cap * sizeof(float), 256);
         const size_t gpan = p.g_vectors ? round_up((size_t)blocks * p.g_vectors * p.g_ld * sizeof(float), 256) : 0;
         if (!ws || !aligned256(ws) || ws_bytes < tri + gpan) return OBC_ERR_WORKSPACE;
