@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 287.8 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 118.9 GB moved for 96.8 GB.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 118.9 / 96.8
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 117.1 GB moved for 96.8 GB.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 117.1 / 96.8
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
