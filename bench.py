@@ -6,9 +6,10 @@ One "step" is one pass of the whole hot path over one layer, through the C ABI:
   final weights (per configuration; see WORKLOADS).
 Prints ONE JSON line.  `value` = eliminated (pruned or quantised) weights per second over the whole job with
 inputs resident in HBM; `e2e` = the same with host<->device copies inside the timed region;
-`roofline` = bytes the elimination kernel has to move per launch over its CUDA-event time, against the measured
-HBM copy rate (for the blocked engine: one read + one write of the active triangle per block of deferred updates;
-the 8 m^2-per-step model of the step-by-step method is reported beside it);
+`roofline` = for the blocked engine the FP32 flops of the deferred updates over the kernel's CUDA-event time against
+the FP32 peak (bound "alu"; the bytes of its schedule against the HBM copy rate are reported beside it), for the
+streaming engine the triangle bytes per step against the measured HBM copy rate (bound "hbm"); the 8 m^2-per-step
+model of the step-by-step method is reported in both cases;
 `cpu_baseline` = the FP64 oracle on a bounded sample of the same rows on this machine's host cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1..C5] [--engine blocked|streaming] [--impl reference]
@@ -381,26 +382,33 @@ def run_ours(args):
     sec = eng_ms * 1e-3
     achieved = own_bytes / sec / 1e9 if sec > 0 else 0.0
     fp32_peak = plan["sm_count"] * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12   # TFLOP/s, FMA = 2
-    roofline = {"bound": "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
-                "achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": round(achieved / peak, 4),
+    hbm = {"achieved": round(achieved, 1), "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+           "frac": round(achieved / peak, 4), "algorithmic_bytes_per_launch": int(own_bytes // n_eng),
+           "bytes_model": ("one write of the private lower triangle, then one read + one write of the compacted "
+                           "triangle per block of deferred updates" if blocked else
+                           "one read + one write of the active lower triangle per step")}
+    tflops = flops / sec / 1e12 if sec > 0 else 0.0
+    alu = {"achieved": round(tflops, 2), "peak": round(fp32_peak, 1), "peak_kind": "derived: SMs x 128 FP32 lanes x 2 x max SM clock",
+           "unit": "TFLOP/s", "frac": round(tflops / fp32_peak, 4), "flops_per_launch": int(flops // n_eng),
+           "flops_model": "2 flops per element of the active lower triangle and update"}
+    # The streaming engine is bound by HBM.  The blocked engine defers updates until its pass over the triangle is
+    # bound by the FP32 FMA work (same flops, ~1/B of the bytes), so its roofline is the ALU one; the HBM figures of
+    # its schedule are kept beside it.
+    main, other = (alu, hbm) if blocked else (hbm, alu)
+    roofline = {"bound": "alu" if blocked else "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
+                "achieved": main["achieved"], "peak": main["peak"], "peak_kind": main["peak_kind"], "unit": main["unit"],
+                "frac": main["frac"],
                 "traffic": int(own_bytes / n_eng * BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE) if blocked
                            else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                "traffic_source": ("scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes" if blocked else
-                                   "scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
-                "algorithmic_bytes_per_launch": int(own_bytes // n_eng), "ms_per_launch": round(eng_ms / n_eng, 3),
-                "launches_timed": len(engine_runs),
-                "bytes_model": ("one write of the private lower triangle, then one read + one write of the compacted "
-                                "triangle per block of deferred updates" if blocked else
-                                "one read + one write of the active lower triangle per step"),
+                "traffic_source": ("DRAM bytes, scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes" if blocked else
+                                   "DRAM bytes, scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
+                "ms_per_launch": round(eng_ms / n_eng, 3), "launches_timed": len(engine_runs),
+                "alu" if blocked else "hbm": main, "hbm" if blocked else "alu": other,
                 "step_by_step_model": {"bytes_per_launch": int(model_bytes // n_eng),
                                        "GBps_equivalent": round(model_bytes / sec / 1e9, 1) if sec > 0 else 0.0,
                                        "over_hbm_peak": round(model_bytes / sec / 1e9 / peak, 3) if sec > 0 else 0.0,
                                        "note": "8 m^2 bytes per elimination step (read + write of the full active block), "
                                                "the figure the step-by-step method has to move"},
-                "alu": {"achieved_tflops": round(flops / sec / 1e12, 2) if sec > 0 else 0.0, "fp32_peak_tflops": round(fp32_peak, 1),
-                        "frac": round(flops / sec / 1e12 / fp32_peak, 4) if sec > 0 else 0.0,
-                        "note": "2 flops per triangle element and update; peak = SMs x 128 FMA lanes x 2 x max SM clock"},
                 "plan": plan}
     if blocked and args.compare_streaming:
         roofline["streaming_engine"] = streaming_reference(layer, peak)
