@@ -1,4 +1,4 @@
-"""Parity at the BASELINE configurations' full sizes, in the launch configuration bench.py times (all rows of the
+"""Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times (all rows of the
 layer in one call), checked on sampled rows the oracle can compute one by one, plus properties that hold at any
 size (every order is a permutation, masks match counts, codes lie on the grid)."""
 import numpy as np

@@ -112,7 +112,7 @@ def test_inverse_reports_non_positive_definite(obc):
 
 # ---------------------------------------------------------------------------------------------------------------
 def test_config1_full_pipeline(obc):
-    """BASELINE config 1: 32x64 layer; full prune trace -> 50% global mask -> weights; 4-bit symmetric OBQ."""
+    """benchmark configuration C1: 32x64 layer; full prune trace -> 50% global mask -> weights; 4-bit symmetric OBQ."""
     W, X, spec = obc_synth.make_layer("C1")
     R, d = W.shape
     H, Hinv = gpu_hinv(obc, X)
@@ -255,7 +255,7 @@ def test_minmax_grid_against_oracle(obc):
 
 
 def test_compound_prune_then_quantize(obc):
-    """BASELINE config 4 in small: global 50% mask from the trace, then 8-bit OBQ on the survivors."""
+    """benchmark configuration C4 in small: global 50% mask from the trace, then 8-bit OBQ on the survivors."""
     W, X, spec = obc_synth.make_layer("C4", n_override=4096)
     rows = 5
     W = W[:rows]
