@@ -406,3 +406,25 @@ def test_pin_block_pruning(c):
     for r in range(2):
         assert np.array_equal(ro["order"][r, ::c] // c, np.argsort(score[r], kind="stable"))
         assert np.allclose(ro["loss"][r, ::c], np.sort(score[r]), rtol=1e-12)
+
+
+def test_golden_c1_trace_is_reproduced():
+    """the stored C1 trace (written by tests/golden/make_c1_trace.py from the oracle alone) is reproduced: guards
+    the oracle's arithmetic against unintended changes"""
+    import importlib.util
+    here = os.path.join(os.path.dirname(__file__), "golden")
+    spec = importlib.util.spec_from_file_location("make_c1_trace", os.path.join(here, "make_c1_trace.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    order, loss, codes, qorder = mod.compute()
+    want = {}
+    for line in open(os.path.join(here, "c1_trace_rows.txt")):
+        if line.startswith("#"):
+            continue
+        name, r, *vals = line.split()
+        want[(name, int(r))] = vals
+    for r in range(3):
+        assert [int(v) for v in want[("order", r)]] == order[r].tolist()
+        assert [int(v) for v in want[("codes", r)]] == codes[r].tolist()
+        assert [int(v) for v in want[("qorder", r)]] == qorder[r].tolist()
+        assert np.allclose([float(v) for v in want[("loss", r)]], loss[r], rtol=1e-12, atol=0)
