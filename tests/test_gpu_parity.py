@@ -472,3 +472,16 @@ def test_prune_blocks_against_oracle(d, rows, kind, threads, max_pending):
         assert np.array_equal(c, oc) and np.array_equal(mk, om)
     finally:
         m.obc_set_engine(m.ENGINE_AUTO)
+
+
+def test_prune_trace_at_maximum_row_length(obc):
+    """d_col = OBC_MAX_DCOL (5120): the first 160 steps of two rows against the oracle (shared memory holds only a
+    few pending vectors at this length, the rest overflow to the L2-resident buffer of the blocked engine)"""
+    d, rows, steps = 5120, 2, 160
+    W, X = obc_synth.make_small(rows, d, d + 512, 5120, "relu")
+    H, Hinv = gpu_hinv(obc, X, prec=obc.PREC_BF16X3)
+    order, loss, status, _ = run_trace(obc, dev(W), Hinv, steps=steps)
+    assert int(status.abs().sum()) == 0
+    o = order.cpu().numpy()
+    assert np.all(o[:, steps:] == -7) and all(len(set(o[r, :steps].tolist())) == steps for r in range(rows))
+    check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), steps=steps)
