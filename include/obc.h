@@ -57,7 +57,7 @@ enum {
 
 typedef enum {
     OBC_OP_HESSIAN = 0, OBC_OP_INVERSE = 1, OBC_OP_PRUNE_TRACE = 2, OBC_OP_SELECT = 3,
-    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5, OBC_OP_PRUNE_BLOCKS = 6
+    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5, OBC_OP_PRUNE_BLOCKS = 6, OBC_OP_CROSS_GRAM = 7
 } obc_op;
 
 /* Which row elimination engine obc_prune_trace / obc_prune_apply / obc_quantize run (all compute Algorithm 1 /
@@ -107,6 +107,19 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n);
 obc_status obc_hessian(const float *X, int d_col, int64_t n, int64_t ldx,
                        float *H, int ldh, int accumulate, obc_prec prec,
                        void *ws, size_t ws_bytes, obc_stream stream);
+
+/* Appendix "Sequential Quantization with OBQ": when the layer inputs X come from the already compressed model, the
+ * dense weights are first re-fitted in closed form, W^T = (X X^T)^-1 X Y^T (Y = the dense model's outputs, d_row x n),
+ * so that they minimise the layer objective again.  X Y^T is accumulated over batches like the Hessian:
+ *   obc_cross_gram : G (+)= Y X^T   (G: d_row x d_col, ldg >= d_col; Y: d_row x n, ldy >= n; X: d_col x n, ldx >= n;
+ *                    prec as in obc_hessian; workspace obc_workspace_bytes(OBC_OP_CROSS_GRAM, d_row, d_col, n))
+ *   obc_refit      : W = 2 G Hinv with Hinv = inv(2 X X^T + lambda I) from obc_hessian / obc_hessian_inverse on the
+ *                    same X, i.e. the least-squares weights with the solver's dampening lambda/2 on X X^T. */
+obc_status obc_cross_gram(const float *Y, int64_t ldy, const float *X, int64_t ldx, int d_row, int d_col, int64_t n,
+                          float *G, int ldg, int accumulate, obc_prec prec,
+                          void *ws, size_t ws_bytes, obc_stream stream);
+obc_status obc_refit(const float *G, int ldg, const float *Hinv, int ldhi, int d_row, int d_col,
+                     float *W_out, int ldwo, obc_stream stream);
 
 /* Section 3 ("Implementation Details"): Hinv = inv(H + damp_rel * mean(diag H) * I) through a Cholesky
  * factorisation carried in FP64, written as an exactly symmetric FP32 matrix (ldhi >= d_col).

@@ -163,6 +163,18 @@ def run_rows_blocks(Hinv, W, c: int, steps=None, forced_blocks=None, return_hi=F
     return out
 
 
+def refit(X, Y, damp_rel: float):
+    """Dense refit before sequential compression (appendix "Sequential Quantization with OBQ"): the closed-form
+    least-squares weights W^T = (X X^T)^-1 X Y^T, with the solver's dampening: W = Y X^T (X X^T + (lambda/2) I)^-1,
+    lambda = damp_rel * mean(diag(2 X X^T)), solved in FP64 with the library's linear solver."""
+    X = np.asarray(X, dtype=np.float64)
+    Y = np.asarray(Y, dtype=np.float64)
+    d = X.shape[0]
+    A = X @ X.T
+    lam = damp_rel * np.trace(2.0 * A) / d
+    return np.linalg.solve(A + 0.5 * lam * np.eye(d), X @ Y.T).T
+
+
 def eliminate_one_row(Hinv, w, **kw):
     """Single-row variant that also returns the row's private Hinv copy after the steps ('Hi')."""
     Hi = np.array(Hinv, dtype=np.float64, order="C", copy=True)

@@ -13,13 +13,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIBPATH = os.path.join(_HERE, "libobc.so")
 
-OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS = range(7)
+OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS, OP_CROSS_GRAM = range(8)
 PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
 FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
+    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_cross_gram", "obc_refit", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -59,6 +59,10 @@ def load_library():
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
     lib.obc_hessian.argtypes = [vp, c_int, c_i64, c_i64, vp, c_int, c_int, c_int, vp, c_sz, vp]
+    lib.obc_cross_gram.restype = c_int
+    lib.obc_cross_gram.argtypes = [vp, c_i64, vp, c_i64, c_int, c_int, c_i64, vp, c_int, c_int, c_int, vp, c_sz, vp]
+    lib.obc_refit.restype = c_int
+    lib.obc_refit.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, c_int, vp]
     lib.obc_hessian_inverse.restype = c_int
     lib.obc_hessian_inverse.argtypes = [vp, c_int, c_int, c_f, vp, c_int, vp, vp, c_sz, vp]
     lib.obc_prune_trace.restype = c_int
@@ -156,6 +160,28 @@ def obc_hessian(X, H, accumulate=False, prec=PREC_FP32, ws=None, stream=None):
     _raise(load_library().obc_hessian(_ptr(X), d, n, _ld(X), _ptr(H), _ld(H), int(bool(accumulate)), int(prec),
                                       _ptr(ws), nb, _stream(stream)), "obc_hessian")
     return H
+
+
+def obc_cross_gram(Y, X, G, accumulate=False, prec=PREC_FP32, ws=None, stream=None):
+    """G (+)= Y X^T for one chunk of the calibration axis (Y: d_row x n dense outputs, X: d_col x n inputs)."""
+    _check(Y, torch.float32, "Y"); _check(X, torch.float32, "X"); _check(G, torch.float32, "G")
+    R, n = Y.shape
+    d = X.shape[0]
+    nb = 0
+    if prec != PREC_FP32:
+        ws, nb = _workspace(ws, OP_CROSS_GRAM, R, d, n, X.device, "obc_cross_gram")
+    _raise(load_library().obc_cross_gram(_ptr(Y), _ld(Y), _ptr(X), _ld(X), R, d, n, _ptr(G), _ld(G), int(bool(accumulate)),
+                                         int(prec), _ptr(ws), nb, _stream(stream)), "obc_cross_gram")
+    return G
+
+
+def obc_refit(G, Hinv, W_out, stream=None):
+    """W_out = 2 G Hinv: the dense least-squares weights for the inputs behind G and Hinv."""
+    _check(G, torch.float32, "G"); _check(Hinv, torch.float32, "Hinv"); _check(W_out, torch.float32, "W_out")
+    R, d = G.shape
+    _raise(load_library().obc_refit(_ptr(G), _ld(G), _ptr(Hinv), _ld(Hinv), R, d, _ptr(W_out), _ld(W_out),
+                                    _stream(stream)), "obc_refit")
+    return W_out
 
 
 def obc_hessian_inverse(H, damp_rel, Hinv=None, info=None, ws=None, stream=None):

@@ -87,6 +87,7 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
         case OBC_OP_HESSIAN: return n > 0 ? hessian_workspace_bytes(d_col, n) : 0;
         case OBC_OP_INVERSE: return inverse_workspace_bytes(d_col);
         case OBC_OP_SELECT: return row_count > 0 ? select_workspace_bytes(row_count, d_col) : 0;
+        case OBC_OP_CROSS_GRAM: return (n > 0 && row_count > 0) ? cross_workspace_bytes(row_count, d_col, n) : 0;
         case OBC_OP_PRUNE_BLOCKS: {
             DeviceInfo di;
             if (device_info(&di) != OBC_OK || d_col > OBC_MAX_DCOL) return 0;
@@ -112,6 +113,28 @@ obc_status obc_hessian(const float* X, int d_col, int64_t n, int64_t ldx, float*
     if (!ws || !aligned256(ws) || ws_bytes < hessian_workspace_bytes(d_col, n)) return OBC_ERR_WORKSPACE;
     if (prec == OBC_PREC_FP32) return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, ws, (cudaStream_t)stream);
     return hessian_tc_launch(X, d_col, n, ldx, H, ldh, accumulate, prec, ws, (cudaStream_t)stream);
+}
+
+obc_status obc_cross_gram(const float* Y, int64_t ldy, const float* X, int64_t ldx, int d_row, int d_col, int64_t n,
+                          float* G, int ldg, int accumulate, obc_prec prec, void* ws, size_t ws_bytes,
+                          obc_stream stream) {
+    if (d_row <= 0 || d_col <= 0 || n <= 0 || !mat_ok(Y, ldy, n) || !mat_ok(X, ldx, n) || !mat_ok(G, ldg, d_col))
+        return OBC_ERR_INVALID_ARG;
+    if (accumulate != 0 && accumulate != 1) return OBC_ERR_INVALID_ARG;
+    if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
+    if (!mat_aligned(Y, ldy) || !mat_aligned(X, ldx)) return OBC_ERR_ALIGNMENT;
+    if (prec == OBC_PREC_FP32)
+        return sgemm_nt_launch(d_row, d_col, n, 1.f, Y, ldy, X, ldx, accumulate ? 1.f : 0.f, G, ldg, (cudaStream_t)stream);
+    if (!ws || !aligned256(ws) || ws_bytes < cross_workspace_bytes(d_row, d_col, n)) return OBC_ERR_WORKSPACE;
+    return cross_tc_launch(Y, d_row, ldy, X, d_col, ldx, n, G, ldg, accumulate, prec, ws, (cudaStream_t)stream);
+}
+
+obc_status obc_refit(const float* G, int ldg, const float* Hinv, int ldhi, int d_row, int d_col, float* W_out, int ldwo,
+                     obc_stream stream) {
+    if (d_row <= 0 || d_col <= 0 || !mat_ok(G, ldg, d_col) || !mat_ok(Hinv, ldhi, d_col) || !mat_ok(W_out, ldwo, d_col))
+        return OBC_ERR_INVALID_ARG;
+    // Hinv is symmetric, so G Hinv = G Hinv^T is the "A B^T" product
+    return sgemm_nt_launch(d_row, d_col, d_col, 2.f, G, ldg, Hinv, ldhi, 0.f, W_out, ldwo, (cudaStream_t)stream);
 }
 
 obc_status obc_hessian_inverse(const float* H, int d_col, int ldh, float damp_rel, float* Hinv, int ldhi,

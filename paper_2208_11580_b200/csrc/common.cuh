@@ -69,6 +69,11 @@ obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, fl
                                void* ws, cudaStream_t stream);
 obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
                              obc_prec prec, void* ws, cudaStream_t stream);
+size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n);
+obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
+                           float* G, int ldg, int accumulate, obc_prec prec, void* ws, cudaStream_t stream);
+obc_status sgemm_nt_launch(int M, int N, int64_t K, float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
+                           float beta, float* C, int ldc, cudaStream_t stream);
 obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const uint8_t* mask, int bits, int symmetric,
                               float* scale, float* zero, cudaStream_t stream);
 obc_status trace_gather_launch(const float* w_trace, int trace_steps, const int32_t* counts, int d, int row_begin,

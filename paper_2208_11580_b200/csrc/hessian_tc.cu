@@ -104,12 +104,18 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t fmt) {
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(TC_TILE >> 3) << 17) | ((uint32_t)(TC_TILE >> 4) << 24);
 }
 
-// KIND 0: TF32, one tensor map (FP32 X).  KIND 1: BF16X3, two maps (hi, lo).
-template <int KIND>
+// KIND 0: TF32, one tensor map per operand (FP32 data).  KIND 1: BF16X3, two maps per operand (hi, lo).
+// CROSS = false: SYRK, both operands are row tiles of the same matrix (maps a == b), lower tile pairs only, d x d
+// output.  CROSS = true: a general A B^T with A rows_a x n (maps a) and B rows_b x n (maps b), all tile pairs,
+// rows_a x rows_b output (used for Y X^T of the dense refit).
+template <int KIND, bool CROSS>
 __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                             const __grid_constant__ CUtensorMap map_lo, int d,
-                                                             int64_t n_elems, int64_t slice, int stages,
-                                                             float* __restrict__ partial, int* __restrict__ err) {
+                                                             const __grid_constant__ CUtensorMap map_lo,
+                                                             const __grid_constant__ CUtensorMap map_b,
+                                                             const __grid_constant__ CUtensorMap map_blo,
+                                                             int rows_a, int rows_b, int64_t n_elems, int64_t slice,
+                                                             int stages, float* __restrict__ partial,
+                                                             int* __restrict__ err) {
     constexpr int TILES_PER_STAGE = KIND == 0 ? 2 : 4;             // A,B (+ A_lo, B_lo)
     constexpr int KELEMS = KIND == 0 ? 32 : 64;                    // elements of K per stage (128 bytes)
     constexpr int KSTEP = KIND == 0 ? 8 : 16;                      // elements of K per MMA (32 bytes)
@@ -119,9 +125,15 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
-    int bi = 0, t = blockIdx.x;
-    while (t > bi) { t -= bi + 1; ++bi; }
-    const int bj = t;
+    int bi = 0, bj = 0;
+    if (CROSS) {
+        const int tj = (rows_b + TC_TILE - 1) / TC_TILE;
+        bi = blockIdx.x / tj; bj = blockIdx.x - bi * tj;
+    } else {
+        int t = blockIdx.x;
+        while (t > bi) { t -= bi + 1; ++bi; }
+        bj = t;
+    }
     const int64_t kb0 = (int64_t)blockIdx.y * slice;
     const int64_t ke = kb0 + slice < n_elems ? kb0 + slice : n_elems;
     const int nkb = ke > kb0 ? (int)((ke - kb0 + KELEMS - 1) / KELEMS) : 0;
@@ -157,10 +169,10 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
             const int x = (int)(kb0 + (int64_t)kb * KELEMS);       // multiple of 128 bytes: satisfies the 16-byte rule
             mbar_expect_tx(full0 + 8 * s, stage_bytes);
             tma_load_2d(dst, &map_a, full0 + 8 * s, x, bi * TC_TILE);
-            tma_load_2d(dst + TC_TILE_BYTES, &map_a, full0 + 8 * s, x, bj * TC_TILE);
+            tma_load_2d(dst + TC_TILE_BYTES, &map_b, full0 + 8 * s, x, bj * TC_TILE);
             if (KIND == 1) {
                 tma_load_2d(dst + 2 * TC_TILE_BYTES, &map_lo, full0 + 8 * s, x, bi * TC_TILE);
-                tma_load_2d(dst + 3 * TC_TILE_BYTES, &map_lo, full0 + 8 * s, x, bj * TC_TILE);
+                tma_load_2d(dst + 3 * TC_TILE_BYTES, &map_blo, full0 + 8 * s, x, bj * TC_TILE);
             }
             issued = kb + 1;
         }
@@ -204,7 +216,7 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
     ab = __shfl_sync(0xffffffffu, ab, 0);
     const bool aborted = !ok || ab != 0;                            // warp-uniform
     if (!aborted) {
-        float* P = partial + (size_t)blockIdx.y * d * d;
+        float* P = partial + (size_t)blockIdx.y * rows_a * rows_b;
         const int gi = bi * TC_TILE + warp * 32 + lane;
         for (int c = 0; c < TC_TILE / 32; ++c) {
             uint32_t r[32];
@@ -213,11 +225,11 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
 #pragma unroll
                 for (int q = 0; q < 32; ++q) r[q] = 0u;
             }
-            if (gi < d) {
+            if (gi < rows_a) {
                 const int gj0 = bj * TC_TILE + c * 32;
 #pragma unroll
                 for (int q = 0; q < 32; ++q)
-                    if (gj0 + q < d) P[(size_t)gi * d + gj0 + q] = __uint_as_float(r[q]);
+                    if (gj0 + q < rows_b) P[(size_t)gi * rows_b + gj0 + q] = __uint_as_float(r[q]);
             }
         }
     }
@@ -315,8 +327,8 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
         ml = ma;
         const int stages = 6;
         const size_t smem = (size_t)stages * 2 * TC_TILE_BYTES + 1024;
-        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<0><<<grid, TC_THREADS, smem, stream>>>(ma, ml, d, n, slice, stages, partial, err);
+        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        syrk_tc_kernel<0, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n, slice, stages, partial, err);
         count_launch();
     } else {
         split_bf16_kernel<<<1184, 256, 0, stream>>>(X, d, n, ldx, n_pad, hi, lo);
@@ -325,12 +337,93 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
         if (!make_map(&ml, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, lo, n_pad, d, n_pad)) return OBC_ERR_CUDA;
         const int stages = 3;
         const size_t smem = (size_t)stages * 4 * TC_TILE_BYTES + 1024;
-        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<1><<<grid, TC_THREADS, smem, stream>>>(ma, ml, d, n_pad, slice, stages, partial, err);
+        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        syrk_tc_kernel<1, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n_pad, slice, stages, partial, err);
         count_launch();
     }
     OBC_CUDA_TRY(cudaGetLastError());
     return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, err, stream);
+}
+
+// ---- G (+)= Y X^T on the tensor cores (appendix "Sequential Quantization with OBQ": X Y^T is accumulated over
+// batches like the Hessian) ------------------------------------------------------------------------------------
+int cross_splits(int rows_a, int rows_b, int64_t n) {
+    const int tiles = ((rows_a + TC_TILE - 1) / TC_TILE) * ((rows_b + TC_TILE - 1) / TC_TILE);
+    int64_t s = (444 + tiles - 1) / tiles;
+    const int64_t by_len = (n + 2047) / 2048;
+    if (by_len > s) s = by_len;
+    if (s > 32) s = 32;
+    if (s * 64 > n) s = n / 64;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n) {
+    const int64_t n_pad = (n + 63) / 64 * 64;
+    return round_up((size_t)cross_splits(rows_a, rows_b, n) * rows_a * rows_b * sizeof(float), 256) + 256 +
+           2 * round_up((size_t)rows_a * n_pad * sizeof(__nv_bfloat16), 256) +
+           2 * round_up((size_t)rows_b * n_pad * sizeof(__nv_bfloat16), 256);
+}
+
+__global__ void __launch_bounds__(256) cross_finalize_kernel(const float* __restrict__ partial, int splits, int rows_a,
+                                                             int rows_b, float* __restrict__ G, int ldg, int accumulate,
+                                                             const int* __restrict__ err) {
+    const int i = blockIdx.y;
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= rows_b) return;
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += partial[(size_t)z * rows_a * rows_b + (size_t)i * rows_b + j];
+    if (accumulate) s += G[(size_t)i * ldg + j];
+    if (err && *err != 0) s = __int_as_float(0x7fc00000);
+    G[(size_t)i * ldg + j] = s;
+}
+
+obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
+                           float* G, int ldg, int accumulate, obc_prec prec, void* ws, cudaStream_t stream) {
+    const int splits = cross_splits(rows_a, rows_b, n);
+    char* p = reinterpret_cast<char*>(ws);
+    float* partial = reinterpret_cast<float*>(p); p += round_up((size_t)splits * rows_a * rows_b * sizeof(float), 256);
+    int* err = reinterpret_cast<int*>(p); p += 256;
+    const int64_t n_pad = (n + 63) / 64 * 64;
+    __nv_bfloat16* yhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up((size_t)rows_a * n_pad * sizeof(__nv_bfloat16), 256);
+    __nv_bfloat16* ylo = reinterpret_cast<__nv_bfloat16*>(p); p += round_up((size_t)rows_a * n_pad * sizeof(__nv_bfloat16), 256);
+    __nv_bfloat16* xhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up((size_t)rows_b * n_pad * sizeof(__nv_bfloat16), 256);
+    __nv_bfloat16* xlo = reinterpret_cast<__nv_bfloat16*>(p);
+    OBC_CUDA_TRY(cudaMemsetAsync(err, 0, sizeof(int), stream));
+    int64_t slice = (n + splits - 1) / splits;
+    slice = (slice + 63) / 64 * 64;
+    const int ti = (rows_a + TC_TILE - 1) / TC_TILE, tj = (rows_b + TC_TILE - 1) / TC_TILE;
+    dim3 grid(ti * tj, splits);
+    CUtensorMap ma, mal, mb, mbl;
+    if (prec == OBC_PREC_TF32) {
+        if (!make_map(&ma, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 4, Y, n, rows_a, ldy)) return OBC_ERR_CUDA;
+        if (!make_map(&mb, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 4, X, n, rows_b, ldx)) return OBC_ERR_CUDA;
+        mal = ma; mbl = mb;
+        const int stages = 6;
+        const size_t smem = (size_t)stages * 2 * TC_TILE_BYTES + 1024;
+        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        syrk_tc_kernel<0, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n, slice, stages, partial, err);
+        count_launch();
+    } else {
+        split_bf16_kernel<<<1184, 256, 0, stream>>>(Y, rows_a, n, ldy, n_pad, yhi, ylo);
+        split_bf16_kernel<<<1184, 256, 0, stream>>>(X, rows_b, n, ldx, n_pad, xhi, xlo);
+        count_launch(2);
+        if (!make_map(&ma, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, yhi, n_pad, rows_a, n_pad)) return OBC_ERR_CUDA;
+        if (!make_map(&mal, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ylo, n_pad, rows_a, n_pad)) return OBC_ERR_CUDA;
+        if (!make_map(&mb, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, xhi, n_pad, rows_b, n_pad)) return OBC_ERR_CUDA;
+        if (!make_map(&mbl, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, xlo, n_pad, rows_b, n_pad)) return OBC_ERR_CUDA;
+        const int stages = 3;
+        const size_t smem = (size_t)stages * 4 * TC_TILE_BYTES + 1024;
+        OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        syrk_tc_kernel<1, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n_pad, slice, stages, partial, err);
+        count_launch();
+    }
+    OBC_CUDA_TRY(cudaGetLastError());
+    dim3 fgrid((rows_b + 255) / 256, rows_a);
+    cross_finalize_kernel<<<fgrid, 256, 0, stream>>>(partial, splits, rows_a, rows_b, G, ldg, accumulate, err);
+    count_launch();
+    OBC_CUDA_TRY(cudaGetLastError());
+    return OBC_OK;
 }
 
 }  // namespace obc

@@ -485,3 +485,30 @@ def test_prune_trace_at_maximum_row_length(obc):
     o = order.cpu().numpy()
     assert np.all(o[:, steps:] == -7) and all(len(set(o[r, :steps].tolist())) == steps for r in range(rows))
     check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), steps=steps)
+
+
+@pytest.mark.parametrize("prec", [0, 1, 2])
+@pytest.mark.parametrize("R,d,n", [(5, 12, 100), (64, 576, 4096), (130, 300, 5000)])
+def test_dense_refit_against_oracle(obc, R, d, n, prec):
+    """dense refit before sequential compression: G = Y X^T (accumulated over two chunks) against FP64, and
+    W = 2 G Hinv against the oracle's regularised least-squares solve"""
+    W0, X = obc_synth.make_small(R, d, n, 2100 + d, "relu")
+    rng = np.random.default_rng(d)
+    Y = (W0.astype(np.float64) @ X.astype(np.float64) + 0.05 * rng.normal(size=(R, n))).astype(np.float32)
+    ldn = (n + 3) // 4 * 4
+    Xd, Yd = padded(X, ldn), padded(Y, ldn)
+    G = torch.zeros(R, (d + 3) // 4 * 4, dtype=torch.float32, device="cuda")[:, :d]
+    h = (n // 2 + 3) // 4 * 4
+    obc.obc_cross_gram(Yd[:, :h], Xd[:, :h], G, accumulate=False, prec=prec)
+    obc.obc_cross_gram(Yd[:, h:], Xd[:, h:], G, accumulate=True, prec=prec)
+    ref = Y.astype(np.float64) @ X.astype(np.float64).T
+    scale = np.sqrt((Y.astype(np.float64) ** 2).sum(axis=1).max() * (X.astype(np.float64) ** 2).sum(axis=1).max())
+    tol = {0: 2e-6, 1: 1e-3, 2: 2e-5}[prec]
+    assert np.abs(G.cpu().numpy() - ref).max() <= tol * scale
+    H, Hinv = gpu_hinv(obc, X, prec=prec)
+    Wn = torch.zeros(R, d, dtype=torch.float32, device="cuda")
+    obc.obc_refit(G, Hinv, Wn)
+    torch.cuda.synchronize()
+    want = oracle.refit(X, Y, DAMP)
+    wtol = {0: 2e-4, 1: 2e-2, 2: 5e-4}[prec]
+    assert np.abs(Wn.cpu().numpy() - want).max() <= wtol * np.abs(want).max()

@@ -428,3 +428,23 @@ def test_golden_c1_trace_is_reproduced():
         assert [int(v) for v in want[("codes", r)]] == codes[r].tolist()
         assert [int(v) for v in want[("qorder", r)]] == qorder[r].tolist()
         assert np.allclose([float(v) for v in want[("loss", r)]], loss[r], rtol=1e-12, atol=0)
+
+
+def test_pin_refit_is_the_regularised_least_squares_optimum():
+    """the dense refit (appendix "Sequential Quantization with OBQ") is the minimiser of ||Y - W X||^2 + (lambda/2)||W||^2:
+    zero gradient, equality with a least-squares solve of the augmented system, and recovery of the generating
+    weights when Y = W0 X exactly and there is no dampening"""
+    rng = np.random.default_rng(3)
+    d, R, n = 11, 4, 90
+    W0, X = obc_synth.make_small(R, d, n, 61)
+    X = X.astype(np.float64)
+    Y = W0.astype(np.float64) @ X + 0.1 * rng.normal(size=(R, n))
+    W = oracle.refit(X, Y, DAMP)
+    lam = DAMP * np.trace(2.0 * X @ X.T) / d
+    grad = -2.0 * (Y - W @ X) @ X.T + lam * W
+    assert np.abs(grad).max() <= 1e-9 * np.abs(2.0 * Y @ X.T).max()
+    X_aug = np.concatenate([X, np.sqrt(lam / 2.0) * np.eye(d)], axis=1)
+    Y_aug = np.concatenate([Y, np.zeros((R, d))], axis=1)
+    sol, *_ = np.linalg.lstsq(X_aug.T, Y_aug.T, rcond=None)
+    assert np.allclose(W, sol.T, rtol=1e-9, atol=1e-12)
+    assert np.allclose(oracle.refit(X, W0.astype(np.float64) @ X, 0.0), W0, rtol=1e-8, atol=1e-10)
