@@ -485,6 +485,8 @@ def test_prune_trace_at_maximum_row_length(obc):
     o = order.cpu().numpy()
     assert np.all(o[:, steps:] == -7) and all(len(set(o[r, :steps].tolist())) == steps for r in range(rows))
     check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), steps=steps)
+    order2, loss2, _, _ = run_trace(obc, dev(W), Hinv, steps=steps)          # a second run is bit-identical
+    assert torch.equal(order, order2) and torch.equal(loss, loss2)
 
 
 @pytest.mark.parametrize("prec", [0, 1, 2])
