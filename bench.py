@@ -237,7 +237,7 @@ class Layer:
         R, d = self.rc, self.d
         key = bool(with_trace)
         if key not in self._info:
-            plan = self.obc.obc_engine_plan(d, with_trace)
+            plan = self.obc.obc_engine_plan(d, with_trace, R)
             info = {"model_bytes": R * model_bytes_full(d), "plan": plan}
             if plan["engine"] == self.obc.ENGINE_BLOCKED:
                 b, f = blocked_bytes_flops(plan, d)
@@ -377,7 +377,7 @@ def run_ours(args):
     own_bytes = sum(i["own_bytes"] for _, _, i in engine_runs)
     model_bytes = sum(i["model_bytes"] for _, _, i in engine_runs)
     flops = sum(i["flops"] for _, _, i in engine_runs)
-    plan = engine_runs[0][2]["plan"] if engine_runs else obc.obc_engine_plan(layer.d)
+    plan = engine_runs[0][2]["plan"] if engine_runs else obc.obc_engine_plan(layer.d, False, layer.rc)
     blocked = plan["engine"] == obc.ENGINE_BLOCKED
     sec = eng_ms * 1e-3
     achieved = own_bytes / sec / 1e9 if sec > 0 else 0.0

@@ -84,15 +84,15 @@ unsigned long long obc_kernel_launches(void);
  * for every choice.  Returns OBC_ERR_INVALID_ARG for values outside these sets. */
 obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
 
-/* How the row engines would run rows of length d_col on the CURRENT device under the present obc_set_engine
- * choice (host function, no launch).  with_trace != 0: as for obc_prune_trace with a weight trace.
+/* How the row engines would run row_count rows (0 = many) of length d_col on the CURRENT device under the present
+ * obc_set_engine choice (host function, no launch).  with_trace != 0: as for obc_prune_trace with a weight trace.
  * plan (host int32[8]): [0] engine (OBC_ENGINE_STREAMING or OBC_ENGINE_BLOCKED), [1] threads per row,
  * [2] rows resident per SM, [3] active size at which a row moves into shared memory, [4] floats of shared memory
  * for deferred update vectors (BLOCKED), [5] limit on deferred updates (BLOCKED), [6] SM count, [7] further
  * deferred update vectors kept in global memory (BLOCKED, long rows; sized to stay in L2).
  * A BLOCKED row of current size m defers min(plan[5], plan[4] / round_up(m, 16) + plan[7]) updates between two
  * passes over its matrix.  Used by the benchmark to state the bytes a launch has to move. */
-obc_status obc_engine_plan(int d_col, int with_trace, int32_t *plan);
+obc_status obc_engine_plan(int d_col, int with_trace, int row_count, int32_t *plan);
 
 /* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).
  * n is only used by OBC_OP_HESSIAN; row_count (the rows one call processes) by the three row-engine ops,

@@ -54,7 +54,7 @@ def load_library():
     lib.obc_set_engine.restype = c_int
     lib.obc_set_engine.argtypes = [c_int, c_int, c_int]
     lib.obc_engine_plan.restype = c_int
-    lib.obc_engine_plan.argtypes = [c_int, c_int, ctypes.POINTER(ctypes.c_int32)]
+    lib.obc_engine_plan.argtypes = [c_int, c_int, c_int, ctypes.POINTER(ctypes.c_int32)]
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
@@ -101,10 +101,10 @@ def obc_set_engine(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int
     _raise(load_library().obc_set_engine(int(engine), int(threads), int(max_pending)), "obc_set_engine")
 
 
-def obc_engine_plan(d_col: int, with_trace: bool = False) -> dict:
-    """How rows of length d_col would run on the current device under the present engine choice."""
+def obc_engine_plan(d_col: int, with_trace: bool = False, row_count: int = 0) -> dict:
+    """How row_count rows (0 = many) of length d_col would run on the current device under the present engine choice."""
     plan = (ctypes.c_int32 * 8)()
-    _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), plan), "obc_engine_plan")
+    _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), int(row_count), plan), "obc_engine_plan")
     return {"engine": int(plan[0]), "threads": int(plan[1]), "rows_per_sm": int(plan[2]), "on_chip_below": int(plan[3]),
             "panel_floats": int(plan[4]), "max_pending": int(plan[5]), "sm_count": int(plan[6]),
             "l2_vectors": int(plan[7])}

@@ -75,10 +75,10 @@ obc_status obc_set_engine(obc_engine engine, int threads, int max_pending) {
     return OBC_OK;
 }
 
-obc_status obc_engine_plan(int d_col, int with_trace, int32_t* plan) {
-    if (d_col <= 0 || !plan) return OBC_ERR_INVALID_ARG;
+obc_status obc_engine_plan(int d_col, int with_trace, int row_count, int32_t* plan) {
+    if (d_col <= 0 || row_count < 0 || !plan) return OBC_ERR_INVALID_ARG;
     if (engine_choice() == OBC_ENGINE_STREAMING) return streaming_engine_plan(d_col, plan);
-    return blocked_engine_plan(d_col, with_trace, plan);
+    return blocked_engine_plan(d_col, with_trace, row_count, plan);
 }
 
 size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {

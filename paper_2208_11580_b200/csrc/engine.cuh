@@ -72,7 +72,7 @@ obc_status streaming_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cuda
 obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream);
 
 obc_status streaming_engine_plan(int d, int32_t* plan);
-obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan);
+obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* plan);
 
 // Process-wide engine choice (see obc_set_engine in obc.h).
 int engine_choice();

@@ -844,10 +844,17 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 
 // Threads per block and blocks per SM by row length: short rows are bound by the latency of a step, so
 // several of them share an SM; long rows need the shared memory for pending vectors.
-static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, bool bc = false) {
+// row_count = rows of the launch (0 = many).
+static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, bool bc = false,
+                     int row_count = 0) {
     const int cap = (d + 3) & ~3;
     int nt = engine_threads_choice();
-    if (nt != 128 && nt != 256 && nt != 512) nt = d <= 512 ? 128 : (d <= 2048 ? 256 : 512);
+    if (nt != 128 && nt != 256 && nt != 512) {
+        // measured on full waves of rows: 128 threads win up to d_col ~ 700, 256 up to ~ 1400, 512 above
+        nt = d <= 704 ? 128 : (d <= 1408 ? 256 : 512);
+        // few rows (one per SM pair at most): nothing to share an SM with, the larger block is faster per row
+        if (nt == 128 && row_count > 0 && row_count <= 2 * di.sm_count) nt = 256;
+    }
     if (nt == 128 && cap > 1024) nt = 256;
     if (nt == 256 && cap > 2048) nt = 512;
     BlkPlan p;
@@ -901,12 +908,12 @@ size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di
            round_up((size_t)gblocks * BLK_MAXB * ((cap + 15) & ~15) * sizeof(float), 256);
 }
 
-obc_status blocked_engine_plan(int d, int with_trace, int32_t* plan) {
+obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* plan) {
     DeviceInfo di;
     obc_status st = device_info(&di);
     if (st != OBC_OK) return st;
     BlkPlan p;
-    if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p)) return OBC_ERR_UNSUPPORTED;
+    if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p, false, false, row_count)) return OBC_ERR_UNSUPPORTED;
     const int mp = engine_pending_choice();
     plan[0] = OBC_ENGINE_BLOCKED; plan[1] = p.nt; plan[2] = p.per_sm; plan[3] = p.ms; plan[4] = p.panel_floats;
     plan[5] = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB; plan[6] = di.sm_count; plan[7] = p.g_vectors;
@@ -939,7 +946,7 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     BlkPlan p;
     const bool bc = a.block_c == 4;
-    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc)) return OBC_ERR_UNSUPPORTED;
+    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc, a.row_count)) return OBC_ERR_UNSUPPORTED;
     a.ms = p.ms;
     a.panel_floats = p.panel_floats;
     int mp = engine_pending_choice();
