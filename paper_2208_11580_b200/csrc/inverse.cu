@@ -16,33 +16,44 @@ constexpr int GK = 16;
 
 // C (MxN) = beta*C + alpha * op(A) (MxK) * op(B) (KxN); row-major doubles.  TA: A is stored KxM.  TB: B is
 // stored NxK.  lower_only: skip tiles strictly above the diagonal (M == N outputs that are symmetric).
+// C may be A itself when N <= GT and A is not transposed: a CTA then reads its own rows completely before it
+// writes them, and no other CTA touches them.
 // k_lo_from_tile: the product only needs k >= max(first row, first column) of the tile (L^-T L^-1).
 template <bool TA, bool TB>
-__device__ __forceinline__ void dgemm_tile(int M, int N, double alpha, const double* __restrict__ A, int lda,
-                                           const double* __restrict__ B, int ldb, double beta, double* __restrict__ C,
+__device__ __forceinline__ void dgemm_tile(int M, int N, double alpha, const double* A, int lda,
+                                           const double* __restrict__ B, int ldb, double beta, double* C,
                                            int ldc, int bm, int bn, int k_begin, int k_end) {
     __shared__ double As[GK][GT + 1];
     __shared__ double Bs[GK][GT + 1];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     double acc[4][4] = {};
-    for (int k0 = k_begin; k0 < k_end; k0 += GK) {
-        for (int e = tid; e < GT * GK; e += 256) {
+    // element e = tid + 256 r of a GT x GK operand tile; the next chunk's elements are fetched into registers
+    // while the current chunk is multiplied
+    double ra[4], rb[4];
+    auto fetch = [&](int k0) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int e = tid + 256 * r;
             int i, k;
             if (TA) { i = e % GT; k = e / GT; } else { k = e % GK; i = e / GK; }
             const int gi = bm + i, gk = k0 + k;
-            double v = 0.0;
-            if (gi < M && gk < k_end) v = TA ? A[(size_t)gk * lda + gi] : A[(size_t)gi * lda + gk];
-            As[k][i] = v;
+            ra[r] = (gi < M && gk < k_end) ? (TA ? A[(size_t)gk * lda + gi] : A[(size_t)gi * lda + gk]) : 0.0;
+            int j, kb;
+            if (TB) { kb = e % GK; j = e / GK; } else { j = e % GT; kb = e / GT; }
+            const int gj = bn + j, gkb = k0 + kb;
+            rb[r] = (gj < N && gkb < k_end) ? (TB ? B[(size_t)gj * ldb + gkb] : B[(size_t)gkb * ldb + gj]) : 0.0;
         }
-        for (int e = tid; e < GT * GK; e += 256) {
-            int j, k;
-            if (TB) { k = e % GK; j = e / GK; } else { j = e % GT; k = e / GT; }
-            const int gj = bn + j, gk = k0 + k;
-            double v = 0.0;
-            if (gj < N && gk < k_end) v = TB ? B[(size_t)gj * ldb + gk] : B[(size_t)gk * ldb + gj];
-            Bs[k][j] = v;
+    };
+    if (k_begin < k_end) fetch(k_begin);
+    for (int k0 = k_begin; k0 < k_end; k0 += GK) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int e = tid + 256 * r;
+            if (TA) As[e / GT][e % GT] = ra[r]; else As[e % GK][e / GK] = ra[r];
+            if (TB) Bs[e % GK][e / GK] = rb[r]; else Bs[e / GT][e % GT] = rb[r];
         }
         __syncthreads();
+        if (k0 + GK < k_end) fetch(k0 + GK);
 #pragma unroll
         for (int k = 0; k < GK; ++k) {
             double a[4], b[4];
@@ -70,9 +81,9 @@ __device__ __forceinline__ void dgemm_tile(int M, int N, double alpha, const dou
 }
 
 template <bool TA, bool TB>
-__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double alpha, const double* __restrict__ A, int lda,
+__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int K, double alpha, const double* A, int lda,
                                                     const double* __restrict__ B, int ldb, double beta,
-                                                    double* __restrict__ C, int ldc, int lower_only, int k_lo_from_tile) {
+                                                    double* C, int ldc, int lower_only, int k_lo_from_tile) {
     const int bm = blockIdx.y * GT, bn = blockIdx.x * GT;
     if (lower_only && bn > bm + GT - 1) return;
     int k0 = 0;
@@ -138,71 +149,96 @@ __global__ void widen_kernel(const float* __restrict__ H, int ldh, int d, const 
 }
 
 // Factor the nb x nb diagonal block at k0 in place (lower Cholesky) and write its inverse into Li.
-__global__ void __launch_bounds__(256) chol_diag_kernel(double* __restrict__ A, double* __restrict__ Li, int d, int k0,
-                                                        int nb, int32_t* info) {
-    __shared__ double L[NB][NB + 1];
-    __shared__ double X[NB][NB + 1];
-    __shared__ int bad;
-    const int tid = threadIdx.x;
-    if (tid == 0) bad = 0;
-    for (int e = tid; e < nb * nb; e += 256) {
-        const int i = e / nb, j = e % nb;
-        L[i][j] = j <= i ? A[(size_t)(k0 + i) * d + k0 + j] : 0.0;
-    }
-    __syncthreads();
-    for (int j = 0; j < nb; ++j) {
-        if (tid == 0) {
-            const double s = L[j][j];
-            if (!(s > 0.0) || !isfinite(s)) { if (!bad) { bad = 1; atomicCAS(info, 0, 1 + k0 + j); } L[j][j] = 1.0; }
-            else L[j][j] = sqrt(s);
+// 16 x 16 threads, each holding a 3 x 3 sub-grid (rows ty + 16p, columns tx + 16q) of the block and of the
+// forward-substitution state S (initially I) in registers.  Column j of the factor is final once columns
+// 0..j-1 have been eliminated, and so is row j of S; one iteration publishes both (unscaled), then every thread
+// applies  A[i][c] -= L[i][j] L[c][j]  and  S[i][c] -= L[i][j] X[j][c]  with  X[j][:] = S[j][:] / L[j][j]
+// to its own elements: one barrier per column (the two publish buffers alternate).  The columns are taken in
+// three groups of 16 (JB), so that which sub-grid elements are above, on or below row / column j is known at
+// compile time except for the group that holds j itself.
+template <int JB>
+__device__ __forceinline__ void chol_diag_columns(double (&a)[3][3], double (&s)[3][3], double (*colL)[NB],
+                                                  double (*rowS)[NB], int nb, int k0, int32_t* info) {
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int jend = min(16, nb - 16 * JB);
+    for (int jl = 0; jl < jend; ++jl) {
+        const int j = 16 * JB + jl;
+        double* cl = colL[jl & 1];
+        double* rs = rowS[jl & 1];
+        if (tx == jl) {
+#pragma unroll
+            for (int p = JB; p < 3; ++p) cl[ty + 16 * p] = a[p][JB];
+        }
+        if (ty == jl) {
+#pragma unroll
+            for (int q = 0; q <= JB; ++q) rs[tx + 16 * q] = s[JB][q];
         }
         __syncthreads();
-        const double ljj = L[j][j];
-        for (int i = j + 1 + tid; i < nb; i += 256) L[i][j] /= ljj;
-        __syncthreads();
-        // trailing update of the block: L[i][c] -= L[i][j] * L[c][j] for j < c <= i
-        const int rem = nb - j - 1;
-        for (int e = tid; e < rem * rem; e += 256) {
-            const int i = j + 1 + e / rem, c = j + 1 + e % rem;
-            if (c <= i) L[i][c] -= L[i][j] * L[c][j];
+        const double piv = cl[j];
+        double ljj = 1.0, inv = 1.0;         // every thread scales by the same reciprocal: FP64 divisions are scarce
+        if (!(piv > 0.0) || !isfinite(piv)) {
+            if (tid == 0) atomicCAS(info, 0, 1 + k0 + j);
+        } else {
+            inv = rsqrt(piv);
+            ljj = piv * inv;
         }
-        __syncthreads();
-    }
-    // X = inv(L): column c solved by thread c (forward substitution)
-    if (tid < nb) {
-        const int c = tid;
-        for (int i = 0; i < nb; ++i) {
-            if (i < c) { X[i][c] = 0.0; continue; }
-            double t = (i == c) ? 1.0 : 0.0;
-            for (int k = c; k < i; ++k) t -= L[i][k] * X[k][c];
-            X[i][c] = t / L[i][i];
+        double li[3], lc[3], xr[3];
+#pragma unroll
+        for (int p = JB; p < 3; ++p) li[p] = cl[ty + 16 * p] * inv;
+#pragma unroll
+        for (int q = JB; q < 3; ++q) lc[q] = cl[tx + 16 * q] * inv;
+#pragma unroll
+        for (int q = 0; q <= JB; ++q) xr[q] = rs[tx + 16 * q] * inv;
+        const bool row_on = ty == jl, row_below = ty > jl, col_on = tx == jl, col_right = tx > jl;
+#pragma unroll
+        for (int p = JB; p < 3; ++p) {
+            const bool below = p > JB || row_below;            // row i > j
+            const bool on = p == JB && row_on;                 // row i == j
+#pragma unroll
+            for (int q = JB; q <= p; ++q) {                    // factor: columns c >= j of rows i >= j
+                const bool right = q > JB || col_right;
+                const bool oncol = q == JB && col_on;
+                if (below && right) a[p][q] = fma(-li[p], lc[q], a[p][q]);
+                else if (below && oncol) a[p][q] = li[p];
+                else if (on && oncol) a[p][q] = ljj;
+            }
+#pragma unroll
+            for (int q = 0; q <= JB; ++q) {                    // substitution: X[j][c] is zero for c > j
+                if (below) s[p][q] = fma(-li[p], xr[q], s[p][q]);
+                else if (on) s[p][q] = xr[q];
+            }
         }
-    }
-    __syncthreads();
-    for (int e = tid; e < nb * nb; e += 256) {
-        const int i = e / nb, j = e % nb;
-        if (j <= i) A[(size_t)(k0 + i) * d + k0 + j] = L[i][j];
-        Li[(size_t)(k0 + i) * d + k0 + j] = X[i][j];
     }
 }
 
-// Panel below the diagonal block: A21 <- A21 * inv(L11)^T, 64 rows per block, in place.
-__global__ void __launch_bounds__(256) chol_panel_kernel(double* __restrict__ A, const double* __restrict__ Li, int d,
-                                                         int k0, int nb) {
-    __shared__ double R[GT][NB + 1];
-    __shared__ double X[NB][NB + 1];
-    const int tid = threadIdx.x;
-    const int i0 = k0 + nb + blockIdx.x * GT;
-    const int rows = min(GT, d - i0);
-    for (int e = tid; e < nb * nb; e += 256) { const int i = e / nb, j = e % nb; X[i][j] = Li[(size_t)(k0 + i) * d + k0 + j]; }
-    for (int e = tid; e < rows * nb; e += 256) { const int i = e / nb, j = e % nb; R[i][j] = A[(size_t)(i0 + i) * d + k0 + j]; }
-    __syncthreads();
-    for (int e = tid; e < rows * nb; e += 256) {
-        const int i = e / nb, j = e % nb;
-        double t = 0.0;
-        for (int k = 0; k <= j; ++k) t += R[i][k] * X[j][k];
-        A[(size_t)(i0 + i) * d + k0 + j] = t;
-    }
+__global__ void __launch_bounds__(256) chol_diag_kernel(double* __restrict__ A, double* __restrict__ Li, int d, int k0,
+                                                        int nb, int32_t* info) {
+    static_assert(NB == 48, "3 x 3 elements per thread of a 16 x 16 thread grid");
+    __shared__ double colL[2][NB];
+    __shared__ double rowS[2][NB];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    double a[3][3], s[3][3];
+#pragma unroll
+    for (int p = 0; p < 3; ++p)
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int i = ty + 16 * p, c = tx + 16 * q;
+            a[p][q] = (i < nb && c <= i) ? A[(size_t)(k0 + i) * d + k0 + c] : 0.0;
+            s[p][q] = i == c ? 1.0 : 0.0;
+        }
+    chol_diag_columns<0>(a, s, colL, rowS, nb, k0, info);
+    if (nb > 16) chol_diag_columns<1>(a, s, colL, rowS, nb, k0, info);
+    if (nb > 32) chol_diag_columns<2>(a, s, colL, rowS, nb, k0, info);
+#pragma unroll
+    for (int p = 0; p < 3; ++p)
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+            const int i = ty + 16 * p, c = tx + 16 * q;
+            if (i < nb && c < nb) {
+                if (c <= i) A[(size_t)(k0 + i) * d + k0 + c] = a[p][q];
+                Li[(size_t)(k0 + i) * d + k0 + c] = c <= i ? s[p][q] : 0.0;
+            }
+        }
 }
 
 // Hinv32[i][j] = Hinv32[j][i] = (float) C[max(i,j)][min(i,j)]
@@ -241,9 +277,9 @@ obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float*
         count_launch();
         const int below = d - k0 - nb;
         if (below > 0) {
-            chol_panel_kernel<<<(below + GT - 1) / GT, 256, 0, s>>>(A, Li, d, k0, nb);
-            count_launch();
-            const double* P = A + (size_t)(k0 + nb) * d + k0;
+            // panel below the diagonal block: A21 <- A21 * inv(L11)^T, in place
+            double* P = A + (size_t)(k0 + nb) * d + k0;
+            dgemm<false, true>(s, below, nb, nb, 1.0, P, d, Li + (size_t)k0 * d + k0, d, 0.0, P, d);
             dgemm<false, true>(s, below, below, nb, -1.0, P, d, P, d, 1.0, A + (size_t)(k0 + nb) * d + k0 + nb, d, 1, 0);
         }
     }
