@@ -121,6 +121,13 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        late = False
+        if not self.rows:          # timed region shorter than the sampling period: take the first sample that arrives
+            late = True
+            for _ in range(30):
+                if self.rows:
+                    break
+                time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -138,8 +145,11 @@ class ClockSampler:
                 pass
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+               "samples": len(sm)}
+        if late:
+            out["note"] = "timed region shorter than the 200 ms sampling period: sample taken right after it"
+        return out
 
 
 # ------------------------------------------------------------------------------------------------------------------

@@ -14,8 +14,9 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The library
- *     allocates nothing, frees nothing and keeps no state between calls.  Scratch memory comes from the
- *     caller's workspace `ws` of at least obc_workspace_bytes(...) bytes (256-byte aligned).
+ *     allocates nothing, frees nothing and keeps no state between calls apart from the process-wide engine
+ *     choice of obc_set_engine.  Scratch memory comes from the caller's workspace `ws` of at least
+ *     obc_workspace_bytes(...) bytes (256-byte aligned).
  *   - Matrices are row-major FP32 with a leading dimension in elements.  Base pointers of FP32 matrices
  *     are 16-byte aligned and leading dimensions are multiples of 4.
  *   - Calls enqueue work on `stream` and return without synchronising.  Argument errors are found on the
