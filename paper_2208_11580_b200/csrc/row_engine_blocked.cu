@@ -38,7 +38,9 @@ constexpr int BLK_OFF_HL = 1792;              // int hl[64]   holes (dead slots 
 constexpr int BLK_OFF_MV = 2048;              // int mv[64]   live slots that move into the holes
 constexpr int BLK_OFF_CM = 2304;
 constexpr int BLK_OFF_RF = 2944;              // float rf[64]  min/max reduction of the compound grid
-constexpr int BLK_FIXED = 3200;
+constexpr int BLK_OFF_GRP = 3200;             // forced groups: int slot[4], float M[4][4] (pivot columns at the pivot slots)
+constexpr int BLK_FIXED = 3328;
+constexpr int BLK_GS = 4;                     // forced eliminations taken together
 
 // Per-row state in shared memory: wd, dg (FP64), perm (int32), srcm (uint16); optional: the row in original
 // order (weight trace), one byte per block of the N:M pattern.
@@ -47,6 +49,9 @@ __host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm =
     return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0) +
            (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0) + (bc ? (size_t)12 * cap : 0);
 }
+// Stride of the pending vectors for a row of m slots: = 8 (mod 32), so that the tensor-core fragments of the
+// flush (4 vectors x 8 consecutive slots per load) touch 32 different banks.
+__host__ __device__ inline int blk_ldz(int m) { return ((m + 8 + 31) & ~31) + 8; }     // >= m + 16
 static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
 
 struct Records {                              // views into one record buffer
@@ -342,6 +347,149 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
     }
 }
 
+// ---- flush on the tensor cores -----------------------------------------------------------------------------------
+// The flush is a rank-nb update, H -= Z^T Z with nb <= 64: a dense contraction.  A warp takes tiles of 16 rows x
+// 64 columns; the increment of a tile is accumulated from zero by mma.sync m16n8k8 (TF32 inputs, FP32
+// accumulation) with every FP32 operand split into two TF32 parts, z = hi + lo, and the three products
+// hi*hi + hi*lo + lo*hi (the missing lo*lo term is below 2^-22 of each product, and the products of one update are
+// about 1/d_col of the element they change).  The tile of H is fetched before the products are formed and arrives
+// meanwhile; the increment is subtracted in FP32 -- one rounding of the matrix element per flush -- and stored.
+// Register layout: lane (g, t) = (lane / 4, lane % 4) holds rows g and g + 8 and, of every 16-column group u, the
+// four columns 16u + 4t .. + 3 (one 128-bit access per row and group).  The two 8-column MMA tiles of a group take
+// its even and its odd columns: tile 2u, n = 2t + e  <->  column 16u + 4t + 2e;  tile 2u+1: that + 1.  Their B
+// fragments (n = g) are then the adjacent pair 16u + 2g, + 1 of a pending vector: one 64-bit shared-memory load.
+// Both parts are rounded to nearest (on the magnitude, ties away): truncation would leave every product short by
+// a part of the same sign, a bias that adds up over the d_col updates of an element instead of averaging out.
+__device__ __forceinline__ uint32_t tf32_rn(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
+__device__ __forceinline__ void tf32_split(float x, uint32_t& hi, uint32_t& lo) {
+    hi = tf32_rn(x);                                        // 11 significant bits
+    lo = tf32_rn(x - __uint_as_float(hi));                  // the difference is exact in FP32
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int NT, bool STREAM>
+__device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, int m1, int nb, const float* Z, int ldz,
+                                              const unsigned short* srcm, const uint32_t* colmask) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int nrg = (m1 + 15) >> 4;
+    const int ksteps = (nb + 7) >> 3;
+    // The products are cheap next to the latency of memory, and a warp has one tile (4 KB) in registers at a time:
+    // a cursor runs FLUSH_AHEAD tiles ahead of the warp through its sequence of tiles and pulls them into L2.
+    constexpr int FLUSH_AHEAD = 4;
+    int prg = warp, pc0 = 0;
+    auto prefetch_next = [&]() {
+        if (prg >= nrg) return;
+        const int row = (prg << 4) + (lane >> 1), col = pc0 + ((lane & 1) << 5);       // 16 rows x 2 lines of 128 bytes
+        if (row < m1 && col <= row)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(Hp + (size_t)srcm[row] * ldp + col));
+        pc0 += 64;
+        if (pc0 >= min((prg << 4) + 16, m1)) { pc0 = 0; prg += NW; }
+    };
+#pragma unroll
+    for (int a = 0; a < FLUSH_AHEAD; ++a) prefetch_next();
+    for (int rg = warp; rg < nrg; rg += NW) {
+        const int i0 = rg << 4;
+        const int jend = min(i0 + 16, m1);                     // columns [0, jend) hold data of this row group
+        const int rr[2] = {i0 + g, i0 + g + 8};                // the lane's two rows
+        const bool in[2] = {rr[0] < m1, rr[1] < m1};
+        const int sr[2] = {in[0] ? (int)srcm[rr[0]] : 0, in[1] ? (int)srcm[rr[1]] : 0};
+        for (int c0 = 0; c0 < jend; c0 += 64) {
+            const int ngroups = min(4, (jend - c0 + 15) >> 4);
+            prefetch_next();
+            float4 hv[4][2];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    hv[u][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const int j = c0 + (u << 4) + (t << 2);
+                    if (u < ngroups && in[h] && j <= rr[h]) {
+                        const float4* src = reinterpret_cast<const float4*>(Hp + (size_t)sr[h] * ldp + j);
+                        hv[u][h] = STREAM ? __ldcs(src) : *src;
+                    }
+                }
+            // columns of this lane that are holes: their data sits in the mover's row (fetched along with the tile)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (u < ngroups) {
+                    const int j = c0 + (u << 4) + (t << 2);
+                    const uint32_t my4 = (colmask[j >> 5] >> (j & 31)) & 0xFu;
+                    if (my4) {
+#pragma unroll
+                        for (int comp = 0; comp < 4; ++comp) {
+                            if (!((my4 >> comp) & 1u)) continue;
+                            const int jj = j + comp;
+                            const int sj = (int)srcm[jj];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                if (in[h] && jj <= rr[h]) {
+                                    const float val = Hp[(size_t)max(sr[h], sj) * ldp + min(sr[h], sj)];
+                                    if (comp == 0) hv[u][h].x = val; else if (comp == 1) hv[u][h].y = val;
+                                    else if (comp == 2) hv[u][h].z = val; else hv[u][h].w = val;
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            float acc[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
+            for (int ks = 0; ks < ksteps; ++ks) {
+                const int k0 = (ks << 3) + t, k1 = k0 + 4;
+                const float* z0 = Z + (size_t)k0 * ldz;
+                const float* z1 = Z + (size_t)k1 * ldz;
+                const bool v0 = k0 < nb, v1 = k1 < nb;
+                uint32_t ah[4], al[4];
+                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
+                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
+                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
+                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (u < ngroups) {
+                        const int c = c0 + (u << 4) + (g << 1);           // < m1 + 16 <= ldz
+                        float2 b0 = make_float2(0.f, 0.f), b1 = b0;
+                        if (v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
+                        if (v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
+                        uint32_t eh0, el0, eh1, el1, oh0, ol0, oh1, ol1;
+                        tf32_split(b0.x, eh0, el0); tf32_split(b1.x, eh1, el1);
+                        tf32_split(b0.y, oh0, ol0); tf32_split(b1.y, oh1, ol1);
+                        mma_tf32(acc[2 * u], al, eh0, eh1);
+                        mma_tf32(acc[2 * u + 1], al, oh0, oh1);
+                        mma_tf32(acc[2 * u], ah, el0, el1);
+                        mma_tf32(acc[2 * u + 1], ah, ol0, ol1);
+                        mma_tf32(acc[2 * u], ah, eh0, eh1);
+                        mma_tf32(acc[2 * u + 1], ah, oh0, oh1);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (u < ngroups) {
+                    const int j = c0 + (u << 4) + (t << 2);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (in[h] && j <= rr[h]) {
+                            float4 o = hv[u][h];
+                            o.x -= acc[2 * u][2 * h];     o.z -= acc[2 * u][2 * h + 1];
+                            o.y -= acc[2 * u + 1][2 * h]; o.w -= acc[2 * u + 1][2 * h + 1];
+                            float4* dst = reinterpret_cast<float4*>(Hp + (size_t)rr[h] * ldp + j);
+                            if (STREAM) __stcs(dst, o); else *dst = o;
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
 // Step-by-step Lemma-1 update on the shared-memory triangle S (leading dimension lds) in the coordinates
 // that hold after slot `last` moved into slot pm (pm < 0: nothing moved); mp = rows left.
 template <int NT>
@@ -383,7 +531,12 @@ __device__ __forceinline__ double block4_score(const double* w, const double* a,
 
 // Q = the kernel contains the OBQ code (modes QUANT and REPLAY_QUANT); the pruning kernels are built without it.
 // BC = 4: block pruning in blocks of 4 consecutive columns (pruning kernels only), 0: single weights.
-template <int NT, int KMAX, bool Q, int BC>
+// FG = the kernel takes forced eliminations (replay of a known order) four at a time: their order is known, so the
+// four pivot columns are fetched and corrected together, the 4 x 4 block of the columns at the pivot slots is
+// broadcast, and every thread carries out the four Lemma-1 eliminations on its own slots in registers -- two
+// barriers per four steps, each pending vector read once for four columns.  Same arithmetic per element as four
+// single steps except that a column's corrections are subtracted one by one instead of summed first.
+template <int NT, int KMAX, bool Q, int BC, bool FG>
 __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
     extern __shared__ __align__(16) char smem[];
     constexpr int NW = NT / 32;
@@ -484,7 +637,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 
         int m0 = d;                      // slots in use (tail phase: number of live slots)
         int nb = 0;                      // pending vectors
-        int ldz = (m0 + 15) & ~15;
+        int ldz = blk_ldz(m0);
         int scap = a.panel_floats / ldz;     // pending vectors that fit into shared memory at this row length
         int bcur = min(a.max_pending, scap + gB);
         if (BC) bcur &= ~(BC - 1);           // whole blocks between two flushes, so that 4-slot groups stay together
@@ -528,7 +681,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         atomicOr(&colmask[h >> 5], 1u << (h & 31));
                     }
                     __syncthreads();
-                    blk_flush<NT, 16, (NT >= 512)>(Hp, ldp, m1, nb, GP ? min(nb, scap) : nb, panel, ldz, G, gld, zstage, srcm, colmask);
+                    if (!GP || nb <= scap)
+                        blk_flush_mma<NT, (NT >= 512)>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
+                    else
+                        blk_flush<NT, 16, (NT >= 512)>(Hp, ldp, m1, nb, min(nb, scap), panel, ldz, G, gld, zstage, srcm, colmask);
                     __syncthreads();
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
@@ -544,7 +700,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     for (int k = 0; k < KMAX; ++k) sa[k] = CUDART_NAN_F;      // slots changed hands: not carried over
 #pragma unroll
                     for (int g = 0; g < KMAX / 4; ++g) cntw[g] = 0u;
-                    ldz = (m0 + 15) & ~15;
+                    ldz = blk_ldz(m0);
                     scap = a.panel_floats / ldz;
                     bcur = min(a.max_pending, scap + gB);
                     if (BC) bcur &= ~(BC - 1);
@@ -562,6 +718,182 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             }
             const bool forced = s < n_forced;
             const bool q_now = Q && quant && !forced;
+            if (FG && forced && !tail && !has_wfull && !has_nm && s + BLK_GS <= n_forced && nb + BLK_GS <= bcur &&
+                (!GP || nb + BLK_GS <= scap)) {
+                // ======================= four forced eliminations together ================================
+                constexpr int GS = BLK_GS;
+                int* gslot = reinterpret_cast<int*>(smem + BLK_OFF_GRP);
+                float* gM = reinterpret_cast<float*>(smem + BLK_OFF_GRP + 16);
+                int fo[GS];
+#pragma unroll
+                for (int g = 0; g < GS; ++g) fo[g] = a.forced_order[(size_t)r * d + s + g];
+                unsigned live = 0u;
+#pragma unroll
+                for (int g4 = 0; g4 < KMAX / 4; ++g4) {
+                    const int jb = own_slot<NT>(4 * g4);
+                    if (jb >= m0) continue;
+                    const int4 pm = *reinterpret_cast<const int4*>(perm + jb);
+                    const int pq[4] = {pm.x, pm.y, pm.z, pm.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (jb + q < m0 && pq[q] >= 0) {
+                            live |= 1u << (4 * g4 + q);
+#pragma unroll
+                            for (int g = 0; g < GS; ++g)
+                                if (pq[q] == fo[g]) gslot[g] = jb + q;
+                        }
+                }
+                __syncthreads();
+                int p4[GS];
+                bool ok = true;
+#pragma unroll
+                for (int g = 0; g < GS; ++g) {
+                    p4[g] = gslot[g];
+                    ok = ok && p4[g] >= 0 && p4[g] < m0 && perm[p4[g]] == fo[g];     // a stale entry never matches
+                }
+                ok = ok && p4[0] != p4[1] && p4[0] != p4[2] && p4[0] != p4[3] && p4[1] != p4[2] && p4[1] != p4[3] &&
+                     p4[2] != p4[3];
+                if (ok) {
+                    double wp4[GS], dp4[GS];
+#pragma unroll
+                    for (int g = 0; g < GS; ++g) { wp4[g] = wd[p4[g]]; dp4[g] = dg[p4[g]]; }
+                    // the four pivot columns of the stored matrix at the own slots
+                    float v[GS][KMAX];
+#pragma unroll
+                    for (int g4 = 0; g4 < KMAX / 4; ++g4) {
+                        const int jb = own_slot<NT>(4 * g4);
+#pragma unroll
+                        for (int g = 0; g < GS; ++g)
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) v[g][4 * g4 + q] = 0.f;
+                        if (jb >= m0) continue;
+#pragma unroll
+                        for (int g = 0; g < GS; ++g) {
+                            const int p = p4[g];
+                            const float* rowp = Hp + (size_t)p * ldp;
+                            if (jb + 3 <= p) {
+                                const float4 t = *reinterpret_cast<const float4*>(rowp + jb);
+                                v[g][4 * g4] = t.x; v[g][4 * g4 + 1] = t.y; v[g][4 * g4 + 2] = t.z; v[g][4 * g4 + 3] = t.w;
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const int j = jb + q;
+                                    if ((live >> (4 * g4 + q)) & 1u) v[g][4 * g4 + q] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                                }
+                            }
+                        }
+                    }
+                    // corrected by the pending vectors (all of them in shared memory here)
+                    for (int b = 0; b < nb; ++b) {
+                        const float* zo = panel + (size_t)b * ldz;
+                        float zp[GS];
+#pragma unroll
+                        for (int g = 0; g < GS; ++g) zp[g] = zo[p4[g]];
+#pragma unroll
+                        for (int g4 = 0; g4 < KMAX / 4; ++g4) {
+                            if ((live >> (4 * g4)) & 0xFu) {
+                                const float4 z = *reinterpret_cast<const float4*>(zo + own_slot<NT>(4 * g4));
+#pragma unroll
+                                for (int g = 0; g < GS; ++g) {
+                                    v[g][4 * g4] = fmaf(-z.x, zp[g], v[g][4 * g4]);
+                                    v[g][4 * g4 + 1] = fmaf(-z.y, zp[g], v[g][4 * g4 + 1]);
+                                    v[g][4 * g4 + 2] = fmaf(-z.z, zp[g], v[g][4 * g4 + 2]);
+                                    v[g][4 * g4 + 3] = fmaf(-z.w, zp[g], v[g][4 * g4 + 3]);
+                                }
+                            }
+                        }
+                    }
+                    // the columns at the four pivot slots, from the owners of those slots
+#pragma unroll
+                    for (int k = 0; k < KMAX; ++k) {
+                        if (!((live >> k) & 1u)) continue;
+                        const int j = own_slot<NT>(k);
+#pragma unroll
+                        for (int g2 = 0; g2 < GS; ++g2)
+                            if (j == p4[g2]) {
+#pragma unroll
+                                for (int g = 0; g < GS; ++g) gM[g * GS + g2] = v[g][k];
+                            }
+                    }
+                    __syncthreads();
+                    // the four eliminations at the pivot slots themselves (every thread, same values)
+                    float zz[GS][GS];                      // vector e at pivot slot x
+                    double idp[GS], fg[GS];
+                    float rsq[GS];
+                    bool fine = true;
+#pragma unroll
+                    for (int g = 0; g < GS; ++g) {
+                        float mc[GS];
+#pragma unroll
+                        for (int x = 0; x < GS; ++x) {
+                            mc[x] = gM[g * GS + x];
+#pragma unroll
+                            for (int e = 0; e < g; ++e) mc[x] = fmaf(-zz[e][x], zz[e][g], mc[x]);
+                        }
+                        const double dpp = dp4[g], w = wp4[g];
+                        if (!(dpp > 0.0) || !isfinite(dpp) || !isfinite(w)) fine = false;
+                        idp[g] = 1.0 / dpp;
+                        fg[g] = w * idp[g];
+                        rsq[g] = __frsqrt_rn((float)dpp);
+#pragma unroll
+                        for (int x = 0; x < GS; ++x) zz[g][x] = mc[x] * rsq[g];
+#pragma unroll
+                        for (int x = g + 1; x < GS; ++x) {
+                            wp4[x] -= fg[g] * (double)mc[x];
+                            dp4[x] -= (double)mc[x] * (double)mc[x] * idp[g];
+                        }
+                    }
+                    if (fine) {
+#pragma unroll
+                        for (int g4 = 0; g4 < KMAX / 4; ++g4) {
+                            const int jb = own_slot<NT>(4 * g4);
+                            if (jb >= m0) continue;
+                            float zv[GS][4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int k = 4 * g4 + q, j = jb + q;
+#pragma unroll
+                                for (int g = 0; g < GS; ++g) zv[g][q] = 0.f;
+                                if (!((live >> k) & 1u)) continue;
+                                int gm = GS;                   // this slot is the gm-th pivot (GS: none of them)
+#pragma unroll
+                                for (int g = 0; g < GS; ++g) if (j == p4[g]) gm = g;
+                                double nw = wd[j], nd = dg[j];
+#pragma unroll
+                                for (int g = 0; g < GS; ++g) {
+                                    if (g < gm) {
+                                        float vj = v[g][k];
+#pragma unroll
+                                        for (int e = 0; e < g; ++e) vj = fmaf(-zv[e][q], zz[e][g], vj);
+                                        nw -= fg[g] * (double)vj;
+                                        nd -= (double)vj * (double)vj * idp[g];
+                                        zv[g][q] = vj * rsq[g];
+                                    }
+                                }
+                                if (gm < GS) perm[j] = -1;
+                                else { wd[j] = nw; dg[j] = nd; }
+                            }
+#pragma unroll
+                            for (int g = 0; g < GS; ++g)
+                                *reinterpret_cast<float4*>(panel + (size_t)(nb + g) * ldz + jb) =
+                                    make_float4(zv[g][0], zv[g][1], zv[g][2], zv[g][3]);
+                        }
+                        if (tid < GS) {
+                            pv[nb + tid] = p4[tid];
+                            if (a.W_out) a.W_out[(size_t)r * a.ldwo + fo[tid]] = 0.f;
+                            if (a.mask) a.mask[(size_t)r * d + fo[tid]] = 0;
+                        }
+                        nb += GS;
+                        s += GS - 1;
+                        sa_valid = false;
+#pragma unroll
+                        for (int k = 0; k < KMAX; ++k) sa[k] = CUDART_NAN_F;
+                        continue;
+                    }
+                }
+                // an entry of the order that is not live, or a pivot that is not positive: the single steps below
+                // meet it again and report it
+            }
             // ---- grid of the compound path: built from the survivors when the replay is over -----------
             if (Q && a.mode == MODE_REPLAY_QUANT && s == n_forced) {
                 float lo = 0.f, hi = 0.f;
@@ -920,11 +1252,11 @@ obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* pl
     return OBC_OK;
 }
 
-template <int NT, int KMAX, bool Q, int BC>
+template <int NT, int KMAX, bool Q, int BC, bool FG>
 static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)smem));
-    blocked_engine_kernel<NT, KMAX, Q, BC><<<blocks, NT, smem, stream>>>(a);
+    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC, FG>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    blocked_engine_kernel<NT, KMAX, Q, BC, FG><<<blocks, NT, smem, stream>>>(a);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
@@ -932,9 +1264,14 @@ static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cud
 
 template <int NT, int KMAX>
 static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    const bool q = a.mode == MODE_QUANT || a.mode == MODE_REPLAY_QUANT;
-    if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4>(a, blocks, smem, stream);
-    return q ? blk_launch_q<NT, KMAX, true, 0>(a, blocks, smem, stream) : blk_launch_q<NT, KMAX, false, 0>(a, blocks, smem, stream);
+    if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4, false>(a, blocks, smem, stream);
+    switch (a.mode) {                       // the replay modes are the ones with forced eliminations
+        case MODE_QUANT:        return blk_launch_q<NT, KMAX, true, 0, false>(a, blocks, smem, stream);
+        // (with 512 threads the OBQ kernel has no registers to spare for the four columns: single steps there)
+        case MODE_REPLAY_QUANT: return blk_launch_q<NT, KMAX, true, 0, (NT <= 256)>(a, blocks, smem, stream);
+        case MODE_REPLAY:       return blk_launch_q<NT, KMAX, false, 0, true>(a, blocks, smem, stream);
+        default:                return blk_launch_q<NT, KMAX, false, 0, false>(a, blocks, smem, stream);
+    }
 }
 static obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream);
 
