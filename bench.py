@@ -52,16 +52,21 @@ def model_bytes_full(d: int, first: int | None = None, steps: int | None = None)
     return int((8.0 * m * m).sum())
 
 
+def pending_stride(m: int) -> int:
+    """Floats between two pending update vectors of a row of m slots (the stride obc_engine_plan documents)."""
+    return (m + 8 + 31) // 32 * 32 + 8
+
+
 def blocked_schedule(plan: dict, first: int, steps: int):
     """(m_after_flush, updates_applied) for every pass the blocked engine makes over a row's matrix when `steps`
-    eliminations start at active size `first`: it defers min(max_pending, panel_floats // round_up(m, 16) + l2_vectors) updates,
-    flushes early when the live size reaches the on-chip threshold, and finishes in shared memory below it."""
+    eliminations start at active size `first`: it defers min(max_pending, panel_floats // pending_stride(m) + l2_vectors)
+    updates, flushes early when the live size reaches the on-chip threshold, and finishes in shared memory below it."""
     ms, panel, maxp = plan["on_chip_below"], plan["panel_floats"], plan["max_pending"]
     out, m0, left = [], first, steps
     if first <= ms:
         return out
     while left > 0 and m0 > ms:
-        b = max(1, min(maxp, panel // ((m0 + 15) // 16 * 16) + plan.get("l2_vectors", 0)))
+        b = max(1, min(maxp, panel // pending_stride(m0) + plan.get("l2_vectors", 0)))
         nb = min(b, m0 - ms, left)
         left -= nb
         if left <= 0:

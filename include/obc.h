@@ -91,8 +91,9 @@ obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
  * [2] rows resident per SM, [3] active size at which a row moves into shared memory, [4] floats of shared memory
  * for deferred update vectors (BLOCKED), [5] limit on deferred updates (BLOCKED), [6] SM count, [7] further
  * deferred update vectors kept in global memory (BLOCKED, long rows; sized to stay in L2).
- * A BLOCKED row of current size m defers min(plan[5], plan[4] / round_up(m, 16) + plan[7]) updates between two
- * passes over its matrix.  Used by the benchmark to state the bytes a launch has to move. */
+ * A BLOCKED row of current size m defers min(plan[5], plan[4] / stride(m) + plan[7]) updates between two passes
+ * over its matrix, stride(m) = round_up(m + 8, 32) + 8 floats per deferred vector.  Used by the benchmark to state
+ * the bytes a launch has to move. */
 obc_status obc_engine_plan(int d_col, int with_trace, int row_count, int32_t *plan);
 
 /* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).

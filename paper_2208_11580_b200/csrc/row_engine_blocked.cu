@@ -349,8 +349,8 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 
 // ---- flush on the tensor cores -----------------------------------------------------------------------------------
 // The flush is a rank-nb update, H -= Z^T Z with nb <= 64: a dense contraction.  A warp takes tiles of 16 rows x
-// 64 columns; the increment of a tile is accumulated from zero by mma.sync m16n8k8 (TF32 inputs, FP32
-// accumulation) with every FP32 operand split into two TF32 parts, z = hi + lo, and the three products
+// 64 columns; the increment of a tile is formed by mma.sync m16n8k8 (TF32 inputs, FP32 accumulation over 8 pending
+// vectors at a time, the partial sums added up in FP32 registers) with every FP32 operand split into two TF32 parts, z = hi + lo, and the three products
 // hi*hi + hi*lo + lo*hi (the missing lo*lo term is below 2^-22 of each product, and the products of one update are
 // about 1/d_col of the element they change).  The tile of H is fetched before the products are formed and arrives
 // meanwhile; the increment is subtracted in FP32 -- one rounding of the matrix element per flush -- and stored.
@@ -446,27 +446,52 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                 const float* z0 = Z + (size_t)k0 * ldz;
                 const float* z1 = Z + (size_t)k1 * ldz;
                 const bool v0 = k0 < nb, v1 = k1 < nb;
-                uint32_t ah[4], al[4];
-                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
-                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
-                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
-                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
+                // all operands of the step first (their latencies overlap), then the products in an order that
+                // puts four independent accumulators between two products into the same one
+                float ar[4];
+                ar[0] = v0 && in[0] ? z0[rr[0]] : 0.f;
+                ar[1] = v0 && in[1] ? z0[rr[1]] : 0.f;
+                ar[2] = v1 && in[0] ? z1[rr[0]] : 0.f;
+                ar[3] = v1 && in[1] ? z1[rr[1]] : 0.f;
+                float2 br[4][2];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    if (u < ngroups) {
-                        const int c = c0 + (u << 4) + (g << 1);           // < m1 + 16 <= ldz
-                        float2 b0 = make_float2(0.f, 0.f), b1 = b0;
-                        if (v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
-                        if (v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
-                        uint32_t eh0, el0, eh1, el1, oh0, ol0, oh1, ol1;
-                        tf32_split(b0.x, eh0, el0); tf32_split(b1.x, eh1, el1);
-                        tf32_split(b0.y, oh0, ol0); tf32_split(b1.y, oh1, ol1);
-                        mma_tf32(acc[2 * u], al, eh0, eh1);
-                        mma_tf32(acc[2 * u + 1], al, oh0, oh1);
-                        mma_tf32(acc[2 * u], ah, el0, el1);
-                        mma_tf32(acc[2 * u + 1], ah, ol0, ol1);
-                        mma_tf32(acc[2 * u], ah, eh0, eh1);
-                        mma_tf32(acc[2 * u + 1], ah, oh0, oh1);
+                    const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
+                    br[u][0] = make_float2(0.f, 0.f);
+                    br[u][1] = make_float2(0.f, 0.f);
+                    if (u < ngroups && v0) br[u][0] = *reinterpret_cast<const float2*>(z0 + c);
+                    if (u < ngroups && v1) br[u][1] = *reinterpret_cast<const float2*>(z1 + c);
+                }
+                uint32_t ah[4], al[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tf32_split(ar[q], ah[q], al[q]);
+#pragma unroll
+                for (int up = 0; up < 4; up += 2) {
+                    if (up < ngroups) {                                   // (a group past the end multiplies zeros)
+                        uint32_t bh[4][2], bl[4][2];                      // tiles 2up .. 2up+3: (k0, k1) parts
+#pragma unroll
+                        for (int w = 0; w < 2; ++w) {
+                            tf32_split(br[up + w][0].x, bh[2 * w][0], bl[2 * w][0]);
+                            tf32_split(br[up + w][1].x, bh[2 * w][1], bl[2 * w][1]);
+                            tf32_split(br[up + w][0].y, bh[2 * w + 1][0], bl[2 * w + 1][0]);
+                            tf32_split(br[up + w][1].y, bh[2 * w + 1][1], bl[2 * w + 1][1]);
+                        }
+                        // The tensor core adds into its accumulator with truncation; over the d_col / 8 steps of an
+                        // element that is a bias.  So the products of one step are summed from zero (small terms
+                        // first) and added to the running increment in FP32 with round-to-nearest.
+                        float dk[4][4];
+#pragma unroll
+                        for (int n = 0; n < 4; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
+#pragma unroll
+                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
+#pragma unroll
+                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
+#pragma unroll
+                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
+#pragma unroll
+                        for (int n = 0; n < 4; ++n)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[2 * up + n][e] += dk[n][e];
                     }
                 }
             }
@@ -1197,7 +1222,7 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     size_t share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
     if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
     const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull, nm, bc);
-    const size_t min_panel = (size_t)4 * ((cap + 15) & ~15);
+    const size_t min_panel = (size_t)4 * blk_ldz(cap);
     while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
         p.per_sm >>= 1;
         share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
@@ -1214,7 +1239,7 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     p.g_ld = (cap + 15) & ~15;
     p.g_vectors = 0;
     if (p.nt == 512) {
-        const int in_smem = p.panel_floats / p.g_ld;
+        const int in_smem = p.panel_floats / blk_ldz(cap);
         int g = (int)(BLK_L2_PANEL_BUDGET / ((size_t)di.sm_count * p.g_ld * 4));
         if (g > 32) g = 32;
         const size_t stage = (size_t)(p.nt / 32) * g * 16 * 4;     // per-warp staging of their row operands
@@ -1292,7 +1317,7 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
         // groups of 4 slots must stay together: no on-chip tail (it compacts slot by slot), whole blocks per flush
         a.ms = 0;
         if (a.max_pending < 4) a.max_pending = 4;
-        if (p.panel_floats / p.g_ld + p.g_vectors < 4) return OBC_ERR_UNSUPPORTED;
+        if (p.panel_floats / blk_ldz(a.cap) + p.g_vectors < 4) return OBC_ERR_UNSUPPORTED;
     }
     int blocks = di.sm_count * p.per_sm;
     if (a.row_count < blocks) blocks = a.row_count;

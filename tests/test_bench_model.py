@@ -13,7 +13,7 @@ def test_blocked_schedule_accounts_for_every_step():
         assert d - sum(nb for _, nb in sched) == sizes[-1] and sizes[-1] <= max(ms, 1) + maxp
         for m1, nb in sched:                     # never more pending updates than fit
             m0 = m1 + nb
-            assert nb <= min(maxp, panel // ((m0 + 15) // 16 * 16) + l2)
+            assert nb <= min(maxp, panel // bench.pending_stride(m0) + l2)
         nbytes, flops = bench.blocked_bytes_flops(plan, d)
         assert nbytes > 2.0 * d * (d + 1) and flops > 0
 
