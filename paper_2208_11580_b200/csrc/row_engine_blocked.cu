@@ -446,35 +446,32 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                 const float* z0 = Z + (size_t)k0 * ldz;
                 const float* z1 = Z + (size_t)k1 * ldz;
                 const bool v0 = k0 < nb, v1 = k1 < nb;
-                // all operands of the step first (their latencies overlap), then the products in an order that
-                // puts four independent accumulators between two products into the same one
-                float ar[4];
-                ar[0] = v0 && in[0] ? z0[rr[0]] : 0.f;
-                ar[1] = v0 && in[1] ? z0[rr[1]] : 0.f;
-                ar[2] = v1 && in[0] ? z1[rr[0]] : 0.f;
-                ar[3] = v1 && in[1] ? z1[rr[1]] : 0.f;
-                float2 br[4][2];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
-                    br[u][0] = make_float2(0.f, 0.f);
-                    br[u][1] = make_float2(0.f, 0.f);
-                    if (u < ngroups && v0) br[u][0] = *reinterpret_cast<const float2*>(z0 + c);
-                    if (u < ngroups && v1) br[u][1] = *reinterpret_cast<const float2*>(z1 + c);
-                }
+                // per pair of column groups: operands first (their latencies overlap), then the products in an order
+                // that puts four independent accumulators between two products into the same one
                 uint32_t ah[4], al[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) tf32_split(ar[q], ah[q], al[q]);
+                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
+                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
+                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
+                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
 #pragma unroll
                 for (int up = 0; up < 4; up += 2) {
                     if (up < ngroups) {                                   // (a group past the end multiplies zeros)
+                        float2 br[2][2];
+#pragma unroll
+                        for (int w = 0; w < 2; ++w) {
+                            const int c = c0 + ((up + w) << 4) + (g << 1);        // < m1 + 16 <= ldz
+                            br[w][0] = make_float2(0.f, 0.f);
+                            br[w][1] = make_float2(0.f, 0.f);
+                            if (up + w < ngroups && v0) br[w][0] = *reinterpret_cast<const float2*>(z0 + c);
+                            if (up + w < ngroups && v1) br[w][1] = *reinterpret_cast<const float2*>(z1 + c);
+                        }
                         uint32_t bh[4][2], bl[4][2];                      // tiles 2up .. 2up+3: (k0, k1) parts
 #pragma unroll
                         for (int w = 0; w < 2; ++w) {
-                            tf32_split(br[up + w][0].x, bh[2 * w][0], bl[2 * w][0]);
-                            tf32_split(br[up + w][1].x, bh[2 * w][1], bl[2 * w][1]);
-                            tf32_split(br[up + w][0].y, bh[2 * w + 1][0], bl[2 * w + 1][0]);
-                            tf32_split(br[up + w][1].y, bh[2 * w + 1][1], bl[2 * w + 1][1]);
+                            tf32_split(br[w][0].x, bh[2 * w][0], bl[2 * w][0]);
+                            tf32_split(br[w][1].x, bh[2 * w][1], bl[2 * w][1]);
+                            tf32_split(br[w][0].y, bh[2 * w + 1][0], bl[2 * w + 1][0]);
+                            tf32_split(br[w][1].y, bh[2 * w + 1][1], bl[2 * w + 1][1]);
                         }
                         // The tensor core adds into its accumulator with truncation; over the d_col / 8 steps of an
                         // element that is a bias.  So the products of one step are summed from zero (small terms
@@ -561,7 +558,8 @@ __device__ __forceinline__ double block4_score(const double* w, const double* a,
 // broadcast, and every thread carries out the four Lemma-1 eliminations on its own slots in registers -- two
 // barriers per four steps, each pending vector read once for four columns.  Same arithmetic per element as four
 // single steps except that a column's corrections are subtracted one by one instead of summed first.
-template <int NT, int KMAX, bool Q, int BC, bool FG>
+// GPV = the kernel can keep further pending vectors in global memory (very long rows, 512 threads only).
+template <int NT, int KMAX, bool Q, int BC, bool FG, bool GPV>
 __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
     extern __shared__ __align__(16) char smem[];
     constexpr int NW = NT / 32;
@@ -597,7 +595,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     const int ldp = a.ldp;
     // overflow of the pending vectors: gB more of them in global memory (sized to stay in L2), stride gld
     // (only the one-row-per-SM configuration uses it; the other kernels are built without that code)
-    constexpr bool GP = NT >= 512;
+    constexpr bool GP = GPV;
     const int gB = (GP && a.Gpan) ? a.g_vectors : 0, gld = a.g_ld;
     float* G = (GP && a.Gpan) ? a.Gpan + (size_t)blockIdx.x * a.g_vectors * a.g_ld : nullptr;
     float* zstage = panel + a.panel_floats + (size_t)warp * a.g_vectors * 16;    // per warp: g_vectors x 16 floats
@@ -1277,14 +1275,20 @@ obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* pl
     return OBC_OK;
 }
 
-template <int NT, int KMAX, bool Q, int BC, bool FG>
-static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC, FG>,
+template <int NT, int KMAX, bool Q, int BC, bool FG, bool GPV>
+static obc_status blk_launch_g(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
+    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    blocked_engine_kernel<NT, KMAX, Q, BC, FG><<<blocks, NT, smem, stream>>>(a);
+    blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV><<<blocks, NT, smem, stream>>>(a);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
+}
+
+template <int NT, int KMAX, bool Q, int BC, bool FG>
+static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
+    if (NT >= 512 && a.Gpan != nullptr) return blk_launch_g<NT, KMAX, Q, BC, FG, (NT >= 512)>(a, blocks, smem, stream);
+    return blk_launch_g<NT, KMAX, Q, BC, FG, false>(a, blocks, smem, stream);
 }
 
 template <int NT, int KMAX>
