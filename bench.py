@@ -6,10 +6,10 @@ One "step" is one pass of the whole hot path over one layer, through the C ABI:
   final weights (per configuration; see WORKLOADS).
 Prints ONE JSON line.  `value` = eliminated (pruned or quantised) weights per second over the whole job with
 inputs resident in HBM; `e2e` = the same with host<->device copies inside the timed region;
-`roofline` = for the blocked engine the FP32 flops of the deferred updates over the kernel's CUDA-event time against
-the FP32 peak (bound "alu"; the bytes of its schedule against the HBM copy rate are reported beside it), for the
-streaming engine the triangle bytes per step against the measured HBM copy rate (bound "hbm"); the 8 m^2-per-step
-model of the step-by-step method is reported in both cases;
+`roofline` = the elimination kernel's bytes over its CUDA-event time against the measured HBM copy rate (bound "hbm"):
+for the blocked engine the bytes of its own schedule (the triangle once per block of deferred updates; the flops of
+the rank-B updates against the TF32 tensor peak are reported beside it), for the streaming engine the triangle bytes
+per step; the 8 m^2-per-step model of the step-by-step method is reported in both cases;
 `cpu_baseline` = the FP64 oracle on a bounded sample of the same rows on this machine's host cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1..C5] [--engine blocked|streaming] [--impl reference]
@@ -34,13 +34,14 @@ import obc_synth  # noqa: E402
 METRIC = "eliminated_weights_per_s"
 UNIT = "weights/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # DRAM bytes per algorithmic byte of the row engine, from the ncu capture summarised in
 # profiles/streaming_engine_d1152_rows148_ncu_full.txt (287.8 GB moved for 603.3 GB of 8 m^2 model bytes); the
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 287.8 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 117.1 GB moved for 96.8 GB.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 117.1 / 96.8
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 122.0 GB moved for 98.1 GB.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 122.0 / 98.1
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
@@ -97,6 +98,17 @@ def peaks():
         j = json.load(open(p))
         return float(j["hbm_gbs"]), "measured"
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def tf32_peak():
+    """Dense TF32 tensor peak in TFLOP/s: the measured sustained bf16 GEMM rate (the kernel runs inside a long step)
+    times the nominal TF32 : BF16 ratio 1.1 : 2.25."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    ratio = 1.1 / 2.25
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return float(j.get("bf16_tflops_sustained", j["bf16_tflops"])) * ratio, "measured sustained bf16 GEMM x 1.1/2.25 (nominal TF32:BF16)"
+    return FALLBACK_BF16_SUSTAINED_TFLOPS * ratio, "fallback sustained bf16 GEMM x 1.1/2.25 (nominal TF32:BF16)"
 
 
 class ClockSampler:
@@ -406,11 +418,20 @@ def run_ours(args):
     alu = {"achieved": round(tflops, 2), "peak": round(fp32_peak, 1), "peak_kind": "derived: SMs x 128 FP32 lanes x 2 x max SM clock",
            "unit": "TFLOP/s", "frac": round(tflops / fp32_peak, 4), "flops_per_launch": int(flops // n_eng),
            "flops_model": "2 flops per element of the active lower triangle and update"}
-    # The streaming engine is bound by HBM.  The blocked engine defers updates until its pass over the triangle is
-    # bound by the FP32 FMA work (same flops, ~1/B of the bytes), so its roofline is the ALU one; the HBM figures of
-    # its schedule are kept beside it.
-    main, other = (alu, hbm) if blocked else (hbm, alu)
-    roofline = {"bound": "alu" if blocked else "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
+    tpeak, tpeak_kind = tf32_peak()
+    tensor = {"achieved": round(tflops, 2), "executed": round(3.0 * tflops, 2), "peak": round(tpeak, 1), "peak_kind": tpeak_kind,
+              "unit": "TFLOP/s", "frac": round(tflops / tpeak, 4), "frac_executed": round(3.0 * tflops / tpeak, 4),
+              "flops_per_launch": int(flops // n_eng),
+              "flops_model": "2 flops per element of the active lower triangle and deferred update (rank-B update on the tensor "
+                             "cores, TF32 m16n8k8); executed = 3 x that: every FP32 operand is split into two TF32 parts and "
+                             "three of the four partial products are formed",
+              "note": "the overflow part of very long rows (d_col > ~2600) still runs as FP32 FMAs"}
+    # Both engines are bound by HBM.  The streaming engine moves the active triangle once per step.  The blocked engine
+    # moves it once per block of deferred updates and applies the block as one rank-B update on the tensor cores, which
+    # costs less than the pass over memory; the per-step phase (argmin, pivot column, correction) moves no matrix bytes
+    # and is inside the same time.
+    main, other = hbm, (tensor if blocked else alu)
+    roofline = {"bound": "hbm", "kernel": "blocked_engine_kernel" if blocked else "row_engine_kernel",
                 "achieved": main["achieved"], "peak": main["peak"], "peak_kind": main["peak_kind"], "unit": main["unit"],
                 "frac": main["frac"],
                 "traffic": int(own_bytes / n_eng * BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE) if blocked
@@ -418,7 +439,7 @@ def run_ours(args):
                 "traffic_source": ("DRAM bytes, scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes" if blocked else
                                    "DRAM bytes, scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
                 "ms_per_launch": round(eng_ms / n_eng, 3), "launches_timed": len(engine_runs),
-                "alu" if blocked else "hbm": main, "hbm" if blocked else "alu": other,
+                "hbm": main, "tensor" if blocked else "alu": other,
                 "step_by_step_model": {"bytes_per_launch": int(model_bytes // n_eng),
                                        "GBps_equivalent": round(model_bytes / sec / 1e9, 1) if sec > 0 else 0.0,
                                        "over_hbm_peak": round(model_bytes / sec / 1e9 / peak, 3) if sec > 0 else 0.0,

@@ -15,8 +15,8 @@
 // vectors and compacts at the same time: a dead slot h below the new size m1 is taken over by a live slot
 // s >= m1, i.e. element (i, j) of the new triangle is read from (max(si, sj), min(si, sj)) of the old one.
 // All such foreign reads come from rows >= m1, which the flush never writes, so it runs in place.
-// The flush works on warp tiles of 16 rows x 128 columns with the 16 x 4 sub-tile of each lane in registers;
-// the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
+// The flush is a rank-B update and runs on the tensor cores (warp tiles of 16 rows x 64 columns, TF32 split
+// products, see blk_flush_mma); the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
 // the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
 // finishes on chip with step-by-step updates.
 //
