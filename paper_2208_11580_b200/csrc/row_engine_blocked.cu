@@ -352,18 +352,20 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 // 64 columns; the increment of a tile is formed by mma.sync m16n8k8 (TF32 inputs, FP32 accumulation over 8 pending
 // vectors at a time, the partial sums added up in FP32 registers) with every FP32 operand split into two TF32 parts, z = hi + lo, and the three products
 // hi*hi + hi*lo + lo*hi (the missing lo*lo term is below 2^-22 of each product, and the products of one update are
-// about 1/d_col of the element they change).  The tile of H is fetched before the products are formed and arrives
-// meanwhile; the increment is subtracted in FP32 -- one rounding of the matrix element per flush -- and stored.
+// about 1/d_col of the element they change).  The tile of H is fetched afterwards (a prefetch cursor has pulled it
+// into L2); the increment is subtracted in FP32 -- one rounding of the matrix element per flush -- and stored.
 // Register layout: lane (g, t) = (lane / 4, lane % 4) holds rows g and g + 8 and, of every 16-column group u, the
 // four columns 16u + 4t .. + 3 (one 128-bit access per row and group).  The two 8-column MMA tiles of a group take
 // its even and its odd columns: tile 2u, n = 2t + e  <->  column 16u + 4t + 2e;  tile 2u+1: that + 1.  Their B
 // fragments (n = g) are then the adjacent pair 16u + 2g, + 1 of a pending vector: one 64-bit shared-memory load.
-// Both parts are rounded to nearest (on the magnitude, ties away): truncation would leave every product short by
-// a part of the same sign, a bias that adds up over the d_col updates of an element instead of averaging out.
+// The leading part is rounded to nearest (on the magnitude, ties away): truncation would leave every product short
+// by a part of the same sign, a bias that adds up over the d_col updates of an element instead of averaging out.
 __device__ __forceinline__ uint32_t tf32_rn(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 __device__ __forceinline__ void tf32_split(float x, uint32_t& hi, uint32_t& lo) {
     hi = tf32_rn(x);                                        // 11 significant bits
-    lo = tf32_rn(x - __uint_as_float(hi));                  // the difference is exact in FP32
+    // the difference is exact in FP32 and has either sign; the tensor core reads its leading 11 bits (truncation of
+    // a part whose sign is random is no bias)
+    lo = __float_as_uint(x - __uint_as_float(hi));
 }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -403,6 +405,56 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
         for (int c0 = 0; c0 < jend; c0 += 64) {
             const int ngroups = min(4, (jend - c0 + 15) >> 4);
             prefetch_next();
+            // ---- the tile's increment: sum over the pending vectors of z[row] * z[column] -------------------------
+            float acc[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
+            for (int ks = 0; ks < ksteps; ks += 2) {
+                // The tensor core adds into its accumulator with truncation; over the d_col / 8 steps of an element
+                // that is a bias.  So the products of 16 pending vectors are summed from zero (small terms first)
+                // and added to the running increment in FP32 with round-to-nearest.  A product into an accumulator
+                // is issued eight products after the previous one into it: their latency is long.
+                float dk[8][4];
+#pragma unroll
+                for (int n = 0; n < 8; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    if (ks + half < ksteps) {
+                        const int k0 = ((ks + half) << 3) + t, k1 = k0 + 4;
+                        const float* z0 = Z + (size_t)k0 * ldz;
+                        const float* z1 = Z + (size_t)k1 * ldz;
+                        const bool v0 = k0 < nb, v1 = k1 < nb;
+                        uint32_t ah[4], al[4];
+                        tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
+                        tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
+                        tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
+                        tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
+                        uint32_t bh[8][2], bl[8][2];                      // the 8 MMA tiles: (k0, k1) parts
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int c = c0 + (u << 4) + (g << 1);       // < m1 + 16 <= ldz
+                            float2 b0 = make_float2(0.f, 0.f), b1 = b0;   // (a group past the end multiplies zeros)
+                            if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
+                            if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
+                            tf32_split(b0.x, bh[2 * u][0], bl[2 * u][0]);
+                            tf32_split(b1.x, bh[2 * u][1], bl[2 * u][1]);
+                            tf32_split(b0.y, bh[2 * u + 1][0], bl[2 * u + 1][0]);
+                            tf32_split(b1.y, bh[2 * u + 1][1], bl[2 * u + 1][1]);
+                        }
+#pragma unroll
+                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
+#pragma unroll
+                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
+#pragma unroll
+                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
+                    }
+                }
+#pragma unroll
+                for (int n = 0; n < 8; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[n][e] += dk[n][e];
+            }
+            // ---- the tile of H (in L2 by now: the cursor passed it two tiles ago), minus the increment -----------
             float4 hv[4][2];
 #pragma unroll
             for (int u = 0; u < 4; ++u)
@@ -415,7 +467,7 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                         hv[u][h] = STREAM ? __ldcs(src) : *src;
                     }
                 }
-            // columns of this lane that are holes: their data sits in the mover's row (fetched along with the tile)
+            // columns of this lane that are holes: their data sits in the mover's row
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 if (u < ngroups) {
@@ -436,60 +488,6 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                                 }
                             }
                         }
-                    }
-                }
-            }
-            float acc[8][4];
-#pragma unroll
-            for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
-            for (int ks = 0; ks < ksteps; ++ks) {
-                const int k0 = (ks << 3) + t, k1 = k0 + 4;
-                const float* z0 = Z + (size_t)k0 * ldz;
-                const float* z1 = Z + (size_t)k1 * ldz;
-                const bool v0 = k0 < nb, v1 = k1 < nb;
-                // per pair of column groups: operands first (their latencies overlap), then the products in an order
-                // that puts four independent accumulators between two products into the same one
-                uint32_t ah[4], al[4];
-                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
-                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
-                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
-                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
-#pragma unroll
-                for (int up = 0; up < 4; up += 2) {
-                    if (up < ngroups) {                                   // (a group past the end multiplies zeros)
-                        float2 br[2][2];
-#pragma unroll
-                        for (int w = 0; w < 2; ++w) {
-                            const int c = c0 + ((up + w) << 4) + (g << 1);        // < m1 + 16 <= ldz
-                            br[w][0] = make_float2(0.f, 0.f);
-                            br[w][1] = make_float2(0.f, 0.f);
-                            if (up + w < ngroups && v0) br[w][0] = *reinterpret_cast<const float2*>(z0 + c);
-                            if (up + w < ngroups && v1) br[w][1] = *reinterpret_cast<const float2*>(z1 + c);
-                        }
-                        uint32_t bh[4][2], bl[4][2];                      // tiles 2up .. 2up+3: (k0, k1) parts
-#pragma unroll
-                        for (int w = 0; w < 2; ++w) {
-                            tf32_split(br[w][0].x, bh[2 * w][0], bl[2 * w][0]);
-                            tf32_split(br[w][1].x, bh[2 * w][1], bl[2 * w][1]);
-                            tf32_split(br[w][0].y, bh[2 * w + 1][0], bl[2 * w + 1][0]);
-                            tf32_split(br[w][1].y, bh[2 * w + 1][1], bl[2 * w + 1][1]);
-                        }
-                        // The tensor core adds into its accumulator with truncation; over the d_col / 8 steps of an
-                        // element that is a bias.  So the products of one step are summed from zero (small terms
-                        // first) and added to the running increment in FP32 with round-to-nearest.
-                        float dk[4][4];
-#pragma unroll
-                        for (int n = 0; n < 4; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
-#pragma unroll
-                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
-#pragma unroll
-                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
-#pragma unroll
-                        for (int n = 0; n < 4; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
-#pragma unroll
-                        for (int n = 0; n < 4; ++n)
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[2 * up + n][e] += dk[n][e];
                     }
                 }
             }
