@@ -409,46 +409,44 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
             float acc[8][4];
 #pragma unroll
             for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
-            for (int ks = 0; ks < ksteps; ks += 2) {
-                // The tensor core adds into its accumulator with truncation; over the d_col / 8 steps of an element
-                // that is a bias.  So the products of 16 pending vectors are summed from zero (small terms first)
-                // and added to the running increment in FP32 with round-to-nearest.  A product into an accumulator
-                // is issued eight products after the previous one into it: their latency is long.
+            for (int ks = 0; ks < ksteps; ++ks) {
+                const int k0 = (ks << 3) + t, k1 = k0 + 4;
+                const float* z0 = Z + (size_t)k0 * ldz;
+                const float* z1 = Z + (size_t)k1 * ldz;
+                const bool v0 = k0 < nb, v1 = k1 < nb;
+                uint32_t ah[4], al[4];
+                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
+                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
+                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
+                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
+                uint32_t bh[8][2], bl[8][2];                              // the 8 MMA tiles: (k0, k1) parts
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
+                    float2 b0 = make_float2(0.f, 0.f), b1 = b0;           // (a group past the end multiplies zeros)
+                    if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
+                    if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
+                    tf32_split(b0.x, bh[2 * u][0], bl[2 * u][0]);
+                    tf32_split(b1.x, bh[2 * u][1], bl[2 * u][1]);
+                    tf32_split(b0.y, bh[2 * u + 1][0], bl[2 * u + 1][0]);
+                    tf32_split(b1.y, bh[2 * u + 1][1], bl[2 * u + 1][1]);
+                }
+                // The tensor core rounds every result toward zero (measured: the products of one instruction are
+                // summed with guard bits, then truncated to FP32).  On a running accumulator that is a bias of about
+                // 2^-25 of the accumulator per instruction, of the same sign for all d_col / 8 instructions of an
+                // element.  So the three products of 8 pending vectors are summed from zero, the two small ones
+                // first -- one truncation at the size of that partial sum -- and the partial sums are added to the
+                // running increment in FP32 with round-to-nearest.  A product into an accumulator is issued eight
+                // products after the previous one into it: their latency is long.
                 float dk[8][4];
 #pragma unroll
                 for (int n = 0; n < 8; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    if (ks + half < ksteps) {
-                        const int k0 = ((ks + half) << 3) + t, k1 = k0 + 4;
-                        const float* z0 = Z + (size_t)k0 * ldz;
-                        const float* z1 = Z + (size_t)k1 * ldz;
-                        const bool v0 = k0 < nb, v1 = k1 < nb;
-                        uint32_t ah[4], al[4];
-                        tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
-                        tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
-                        tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
-                        tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
-                        uint32_t bh[8][2], bl[8][2];                      // the 8 MMA tiles: (k0, k1) parts
+                for (int n = 0; n < 8; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int c = c0 + (u << 4) + (g << 1);       // < m1 + 16 <= ldz
-                            float2 b0 = make_float2(0.f, 0.f), b1 = b0;   // (a group past the end multiplies zeros)
-                            if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
-                            if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
-                            tf32_split(b0.x, bh[2 * u][0], bl[2 * u][0]);
-                            tf32_split(b1.x, bh[2 * u][1], bl[2 * u][1]);
-                            tf32_split(b0.y, bh[2 * u + 1][0], bl[2 * u + 1][0]);
-                            tf32_split(b1.y, bh[2 * u + 1][1], bl[2 * u + 1][1]);
-                        }
+                for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
 #pragma unroll
-                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
-#pragma unroll
-                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
-#pragma unroll
-                        for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
-                    }
-                }
+                for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
 #pragma unroll
                 for (int n = 0; n < 8; ++n)
 #pragma unroll

@@ -373,6 +373,56 @@ def test_blocked_engine_block_sizes(threads, max_pending, d, rows):
         m.obc_set_engine(m.ENGINE_AUTO)
 
 
+@pytest.mark.parametrize("threads,max_pending,d,rows", [(0, 0, 300, 9), (128, 0, 520, 9), (256, 7, 520, 9), (256, 64, 1100, 6),
+                                                        (512, 0, 1100, 6), (512, 5, 300, 9)])
+def test_forced_replay_against_trace_and_oracle(threads, max_pending, d, rows):
+    """forced-order replay (obc_prune_apply without a trace) on rows long enough to run off chip, where the blocked
+    engine takes the forced eliminations four at a time: per-row counts from 0 to d_col, against the GPU's own trace,
+    the oracle's trace, and -- for an order that names a column twice -- the reported status"""
+    import paper_2208_11580_b200 as m
+    m.load_library()
+    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
+    try:
+        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 4100 + d, "relu")
+        H = oracle.hessian(X).astype(np.float32)
+        ld = (d + 3) // 4 * 4
+        Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
+        Wd = padded(W, ld)
+        order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
+        assert int(status.abs().sum()) == 0
+        st = check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
+        cnt = np.array([0, 1, 3, 4, 5, d // 2 + 1, d - 1, d, 37][:rows], dtype=np.int32)
+        counts = torch.from_numpy(cnt).cuda()
+        rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
+        got = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        m.obc_prune_apply(Wd, Hinv, order, counts, got, rs)
+        ref = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        m.obc_prune_apply(Wd, Hinv, order, counts, ref, rs, w_trace=trace, trace_steps=d)
+        torch.cuda.synchronize()
+        assert int(rs.abs().sum()) == 0
+        g, r = got.cpu().numpy(), ref.cpu().numpy()
+        wscale = np.abs(W).max(axis=1, keepdims=True)
+        assert (np.abs(g - r) / wscale).max() <= REL_TOL
+        want = oracle.weights_from_trace(st["oracle"]["w_trace"], cnt)
+        assert (np.abs(g - want) / wscale).max() <= REL_TOL
+        o = order.cpu().numpy()
+        for i in range(rows):
+            assert np.all(g[i, o[i, :cnt[i]]] == 0.0)
+        # an order that is not a permutation: row 5 names its first column again at step 6
+        bad = order.clone()
+        bad[5, 6] = bad[5, 0]
+        rs2 = torch.zeros(rows, dtype=torch.int32, device="cuda")
+        out2 = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        m.obc_prune_apply(Wd, Hinv, bad, counts, out2, rs2)
+        torch.cuda.synchronize()
+        r2 = rs2.cpu().numpy()
+        assert r2[5] == 1 + 6 and np.all(np.delete(r2, 5) == 0)
+        assert np.array_equal(np.delete(out2.cpu().numpy(), 5, axis=0), np.delete(g, 5, axis=0))
+    finally:
+        m.obc_set_engine(m.ENGINE_AUTO)
+
+
+
 def test_sharded_layer_driver_single_rank(obc):
     """the row-sharded layer driver with one rank (no process group): same masks and weights as the oracle"""
     from paper_2208_11580_b200.sharding import prune_layer_sharded
