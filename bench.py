@@ -36,9 +36,9 @@ UNIT = "weights/s"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # DRAM bytes per algorithmic byte of the row engine, from the ncu capture summarised in
-# profiles/streaming_engine_d1152_rows148_ncu_full.txt (287.8 GB moved for 603.3 GB of 8 m^2 model bytes); the
+# profiles/streaming_engine_d1152_rows148_ncu_full.txt (291.0 GB moved for 603.3 GB of 8 m^2 model bytes); the
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
-ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 287.8 / 603.3
+ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 291.0 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
 # profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.3 GB moved for 98.1 GB.
 BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.3 / 98.1
