@@ -40,8 +40,8 @@ FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 291.0 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.3 GB moved for 98.1 GB.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.3 / 98.1
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.1 GB moved for 98.1 GB.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.1 / 98.1
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:

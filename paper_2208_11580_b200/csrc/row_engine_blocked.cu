@@ -649,12 +649,16 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 const float4* s4 = reinterpret_cast<const float4*>(a.Hinv + (size_t)i * a.ldhi);
                 float4* d4 = reinterpret_cast<float4*>(Hp + (size_t)i * ldp);
                 const int n4 = (i >> 2) + 1;
-                for (int j0 = lane; j0 < n4; j0 += 128) {      // four loads in flight per lane
-                    float4 t[4];
+                if (GP || (FG && NT >= 512)) {      // (kernels with no registers to spare: one load in flight)
+                    for (int j4 = lane; j4 < n4; j4 += 32) d4[j4] = s4[j4];
+                } else {
+                    for (int j0 = lane; j0 < n4; j0 += 128) {      // four loads in flight per lane
+                        float4 t[4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) if (j0 + 32 * k < n4) t[k] = __ldg(s4 + j0 + 32 * k);
+                        for (int k = 0; k < 4; ++k) if (j0 + 32 * k < n4) t[k] = __ldg(s4 + j0 + 32 * k);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) if (j0 + 32 * k < n4) d4[j0 + 32 * k] = t[k];
+                        for (int k = 0; k < 4; ++k) if (j0 + 32 * k < n4) d4[j0 + 32 * k] = t[k];
+                    }
                 }
             }
         }
