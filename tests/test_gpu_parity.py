@@ -374,7 +374,7 @@ def test_blocked_engine_block_sizes(threads, max_pending, d, rows):
 
 
 @pytest.mark.parametrize("threads,max_pending,d,rows", [(0, 0, 300, 9), (128, 0, 520, 9), (256, 7, 520, 9), (256, 64, 1100, 6),
-                                                        (512, 0, 1100, 6), (512, 5, 300, 9)])
+                                                        (512, 0, 1100, 6), (512, 5, 300, 9), (0, 0, 301, 9), (256, 0, 519, 7)])
 def test_forced_replay_against_trace_and_oracle(threads, max_pending, d, rows):
     """forced-order replay (obc_prune_apply without a trace) on rows long enough to run off chip, where the blocked
     engine takes the forced eliminations four at a time: per-row counts from 0 to d_col, against the GPU's own trace,
