@@ -712,7 +712,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     }
                     __syncthreads();
                     if (!GP || nb <= scap)
-                        blk_flush_mma<NT, (NT >= 512)>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);
+                        blk_flush_mma<NT, true>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);      // evict-first at every row length (~1 %)
                     else
                         blk_flush<NT, 16, (NT >= 512)>(Hp, ldp, m1, nb, min(nb, scap), panel, ldz, G, gld, zstage, srcm, colmask);
                     __syncthreads();
