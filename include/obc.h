@@ -14,9 +14,9 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The library
- *     allocates nothing, frees nothing and keeps no state between calls apart from the process-wide engine
- *     choice of obc_set_engine.  Scratch memory comes from the caller's workspace `ws` of at least
- *     obc_workspace_bytes(...) bytes (256-byte aligned).
+ *     allocates nothing, frees nothing and keeps no state between calls (the kernel-launch counter of
+ *     obc_kernel_launches is a diagnostic only).  Scratch memory comes from the caller's workspace `ws` of at
+ *     least obc_workspace_bytes(...) bytes (256-byte aligned).
  *   - Matrices are row-major FP32 with a leading dimension in elements.  Base pointers of FP32 matrices
  *     are 16-byte aligned and leading dimensions are multiples of 4.
  *   - Calls enqueue work on `stream` and return without synchronising.  Argument errors are found on the
@@ -78,15 +78,25 @@ const char *obc_status_string(obc_status s);
 /* Diagnostic (host function): number of kernels this library has launched in the calling process so far. */
 unsigned long long obc_kernel_launches(void);
 
-/* Process-wide engine selection (host function; takes effect for calls made after it returns; not meant to be
- * changed while another thread is inside a library call).  threads: threads per row of the BLOCKED engine
- * (128, 256, 512; 0 = chosen from d_col).  max_pending: upper limit on the number of deferred updates
- * (1..64; 0 = as many as the shared memory holds).  Workspace sizes reported by obc_workspace_bytes are valid
- * for every choice.  Returns OBC_ERR_INVALID_ARG for values outside these sets. */
-obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
+/* Per-call choice of how the row elimination engine runs (HOST struct, read before the call returns).  Every
+ * row-engine entry point takes a pointer to one; NULL means all defaults.  Nothing here changes results beyond the
+ * order of FP32 roundings: every choice computes Algorithm 1 / Algorithm 3.
+ *   engine      : a value of the obc_engine enum, AUTO = BLOCKED.  obc_prune_nm / obc_prune_blocks always run BLOCKED and ignore it.
+ *   threads     : BLOCKED engine, threads per row: 128, 256, 512, or 0 = chosen from d_col and row_count.
+ *   max_pending : BLOCKED engine, upper limit on the number of deferred updates, 1..64, or 0 = as many as the
+ *                 shared memory holds.
+ *   reserved    : must be 0.
+ * Values outside these sets make the call return OBC_ERR_INVALID_ARG.  Workspace sizes reported by
+ * obc_workspace_bytes are valid for every choice. */
+typedef struct {
+    int32_t engine;
+    int32_t threads;
+    int32_t max_pending;
+    int32_t reserved;
+} obc_engine_opts;
 
-/* How the row engines would run row_count rows (0 = many) of length d_col on the CURRENT device under the present
- * obc_set_engine choice (host function, no launch).  with_trace != 0: as for obc_prune_trace with a weight trace.
+/* How the row engines would run row_count rows (0 = many) of length d_col on the CURRENT device with the options
+ * `opts` (host function, no launch).  with_trace != 0: as for obc_prune_trace with a weight trace.
  * plan (host int32[8]): [0] engine (OBC_ENGINE_STREAMING or OBC_ENGINE_BLOCKED), [1] threads per row,
  * [2] rows resident per SM, [3] active size at which a row moves into shared memory, [4] floats of shared memory
  * for deferred update vectors (BLOCKED), [5] limit on deferred updates (BLOCKED), [6] SM count, [7] further
@@ -94,7 +104,7 @@ obc_status obc_set_engine(obc_engine engine, int threads, int max_pending);
  * A BLOCKED row of current size m defers min(plan[5], plan[4] / stride(m) + plan[7]) updates between two passes
  * over its matrix, stride(m) = round_up(m + 8, 32) + 8 floats per deferred vector.  Used by the benchmark to state
  * the bytes a launch has to move. */
-obc_status obc_engine_plan(int d_col, int with_trace, int row_count, int32_t *plan);
+obc_status obc_engine_plan(int d_col, int with_trace, int row_count, const obc_engine_opts *opts, int32_t *plan);
 
 /* Bytes of workspace the given call needs for these sizes on the CURRENT device (host function, no launch).
  * n is only used by OBC_OP_HESSIAN; row_count (the rows one call processes) by the three row-engine ops,
@@ -143,7 +153,7 @@ obc_status obc_hessian_inverse(const float *H, int d_col, int ldh, float damp_re
 obc_status obc_prune_trace(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float *Hinv, int ldhi, int steps,
                            int32_t *order, float *loss, float *w_trace, int32_t *row_status,
-                           void *ws, size_t ws_bytes, obc_stream stream);
+                           void *ws, size_t ws_bytes, const obc_engine_opts *opts, obc_stream stream);
 
 /* Section 3, "N:M Sparsity": Algorithm 1 with the argmin restricted to weights whose block of m_block consecutive
  * columns has lost fewer than m_block - n_keep weights so far; after d_col * (m_block - n_keep) / m_block
@@ -159,7 +169,7 @@ obc_status obc_prune_trace(const float *W, int ldw, int d_row, int d_col, int ro
 obc_status obc_prune_nm(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                         const float *Hinv, int ldhi, int n_keep, int m_block,
                         int32_t *order, float *loss, float *W_out, int ldwo, uint8_t *mask, int32_t *row_status,
-                        void *ws, size_t ws_bytes, obc_stream stream);
+                        void *ws, size_t ws_bytes, const obc_engine_opts *opts, obc_stream stream);
 
 /* Section 3, "Block-Sparsity" (Eq. 5): Algorithm 1 on blocks of `block` consecutive columns.  Each step removes the
  * remaining block P with the smallest w_P^T ((Hinv)_P)^-1 w_P (ties: lowest block), compensates the other weights by
@@ -174,7 +184,7 @@ obc_status obc_prune_nm(const float *W, int ldw, int d_row, int d_col, int row_b
 obc_status obc_prune_blocks(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                             const float *Hinv, int ldhi, int block,
                             int32_t *order, float *loss, float *w_trace, int32_t *row_status,
-                            void *ws, size_t ws_bytes, obc_stream stream);
+                            void *ws, size_t ws_bytes, const obc_engine_opts *opts, obc_stream stream);
 
 /* Algorithm 2 (appendix, "ExactOBS Global Step"): repeatedly prune, across all rows, the weight whose
  * next recorded loss is smallest (ties: lowest row), k times.  k is a count, 0 <= k <= d_row*d_col.
@@ -210,7 +220,7 @@ obc_status obc_prune_apply(const float *W, int ldw, int d_row, int d_col, int ro
                            const float *Hinv, int ldhi, const int32_t *order, const int32_t *counts,
                            const float *w_trace, int trace_steps,
                            float *W_out, int ldwo, int32_t *row_status,
-                           void *ws, size_t ws_bytes, obc_stream stream);
+                           void *ws, size_t ws_bytes, const obc_engine_opts *opts, obc_stream stream);
 
 /* Per-row uniform grid over the kept entries (mask NULL = all kept); the range always contains 0.
  *   asymmetric: maxq = 2^bits-1, scale = (hi-lo)/maxq, zero = rne(-lo/scale)
@@ -236,7 +246,7 @@ obc_status obc_quantize(const float *W, int ldw, int d_row, int d_col, int row_b
                         const float *Hinv, int ldhi, float *scale, float *zero, int bits, int symmetric,
                         const int32_t *prune_order, const int32_t *prune_counts, int flags,
                         float *W_out, int ldwo, int32_t *codes, float *loss, int32_t *qorder,
-                        int32_t *row_status, void *ws, size_t ws_bytes, obc_stream stream);
+                        int32_t *row_status, void *ws, size_t ws_bytes, const obc_engine_opts *opts, obc_stream stream);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,7 @@ FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
 
 EXPORTED_SYMBOLS = (
-    "obc_status_string", "obc_kernel_launches", "obc_set_engine", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_cross_gram", "obc_refit", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
+    "obc_status_string", "obc_kernel_launches", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_cross_gram", "obc_refit", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
     "obc_select_global_mask", "obc_select_global_mask_static", "obc_prune_apply", "obc_minmax_grid", "obc_quantize",
 )
 
@@ -51,10 +51,8 @@ def load_library():
     lib.obc_status_string.argtypes = [c_int]
     lib.obc_kernel_launches.restype = ctypes.c_ulonglong
     lib.obc_kernel_launches.argtypes = []
-    lib.obc_set_engine.restype = c_int
-    lib.obc_set_engine.argtypes = [c_int, c_int, c_int]
     lib.obc_engine_plan.restype = c_int
-    lib.obc_engine_plan.argtypes = [c_int, c_int, c_int, ctypes.POINTER(ctypes.c_int32)]
+    lib.obc_engine_plan.argtypes = [c_int, c_int, c_int, vp, ctypes.POINTER(ctypes.c_int32)]
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
@@ -66,24 +64,24 @@ def load_library():
     lib.obc_hessian_inverse.restype = c_int
     lib.obc_hessian_inverse.argtypes = [vp, c_int, c_int, c_f, vp, c_int, vp, vp, c_sz, vp]
     lib.obc_prune_trace.restype = c_int
-    lib.obc_prune_trace.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+    lib.obc_prune_trace.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp, vp]
     lib.obc_prune_nm.restype = c_int
     lib.obc_prune_nm.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, c_int, vp, vp, vp, c_int, vp, vp,
-                                 vp, c_sz, vp]
+                                 vp, c_sz, vp, vp]
     lib.obc_prune_blocks.restype = c_int
-    lib.obc_prune_blocks.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+    lib.obc_prune_blocks.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, vp, vp, vp, c_sz, vp, vp]
     lib.obc_select_global_mask.restype = c_int
     lib.obc_select_global_mask.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp, c_sz, vp]
     lib.obc_select_global_mask_static.restype = c_int
     lib.obc_select_global_mask_static.argtypes = [vp, vp, c_int, c_int, c_i64, vp, vp, vp]
     lib.obc_prune_apply.restype = c_int
     lib.obc_prune_apply.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, vp, vp, vp, c_int, vp, c_int, vp,
-                                    vp, c_sz, vp]
+                                    vp, c_sz, vp, vp]
     lib.obc_minmax_grid.restype = c_int
     lib.obc_minmax_grid.argtypes = [vp, c_int, c_int, c_int, vp, c_int, c_int, vp, vp, ctypes.POINTER(c_int), vp]
     lib.obc_quantize.restype = c_int
     lib.obc_quantize.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, c_int, vp, vp, c_int, c_int, vp, vp, c_int,
-                                 vp, c_int, vp, vp, vp, vp, vp, c_sz, vp]
+                                 vp, c_int, vp, vp, vp, vp, vp, c_sz, vp, vp]
     _lib = lib
     return lib
 
@@ -96,15 +94,30 @@ def obc_kernel_launches() -> int:
     return int(load_library().obc_kernel_launches())
 
 
-def obc_set_engine(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0) -> None:
-    """Process-wide choice of the row elimination engine (streaming rank-1 passes or deferred block updates)."""
-    _raise(load_library().obc_set_engine(int(engine), int(threads), int(max_pending)), "obc_set_engine")
+class EngineOpts(ctypes.Structure):
+    """obc_engine_opts: per-call choice of the row elimination engine (engine, threads per row, limit on deferred
+    updates); all zero = the library's defaults."""
+    _fields_ = [("engine", ctypes.c_int32), ("threads", ctypes.c_int32), ("max_pending", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
-def obc_engine_plan(d_col: int, with_trace: bool = False, row_count: int = 0) -> dict:
-    """How row_count rows (0 = many) of length d_col would run on the current device under the present engine choice."""
+def engine_opts(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0) -> EngineOpts:
+    return EngineOpts(int(engine), int(threads), int(max_pending), 0)
+
+
+def _opts(opts):
+    """None, an EngineOpts, or a (engine, threads, max_pending) tuple -> pointer argument (kept alive by the caller)."""
+    if opts is None:
+        return None
+    if not isinstance(opts, EngineOpts):
+        opts = engine_opts(*opts)
+    return ctypes.cast(ctypes.pointer(opts), ctypes.c_void_p)
+
+
+def obc_engine_plan(d_col: int, with_trace: bool = False, row_count: int = 0, opts=None) -> dict:
+    """How row_count rows (0 = many) of length d_col would run on the current device with the engine options `opts`."""
     plan = (ctypes.c_int32 * 8)()
-    _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), int(row_count), plan), "obc_engine_plan")
+    _raise(load_library().obc_engine_plan(int(d_col), int(bool(with_trace)), int(row_count), _opts(opts), plan), "obc_engine_plan")
     return {"engine": int(plan[0]), "threads": int(plan[1]), "rows_per_sm": int(plan[2]), "on_chip_below": int(plan[3]),
             "panel_floats": int(plan[4]), "max_pending": int(plan[5]), "sm_count": int(plan[6]),
             "l2_vectors": int(plan[7])}
@@ -199,7 +212,7 @@ def obc_hessian_inverse(H, damp_rel, Hinv=None, info=None, ws=None, stream=None)
 
 
 def obc_prune_trace(W, Hinv, order, loss, row_status, steps=None, w_trace=None, row_begin=0, row_count=None,
-                    ws=None, stream=None):
+                    ws=None, opts=None, stream=None):
     """Algorithm 1 on rows [row_begin, row_begin+row_count): fills order, loss (and w_trace)."""
     _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(order, torch.int32, "order")
     _check(loss, torch.float32, "loss"); _check(row_status, torch.int32, "row_status"); _check(w_trace, torch.float32, "w_trace")
@@ -209,11 +222,11 @@ def obc_prune_trace(W, Hinv, order, loss, row_status, steps=None, w_trace=None, 
     ws, nb = _workspace(ws, OP_PRUNE_TRACE, row_count, d, 0, W.device, "obc_prune_trace")
     _raise(load_library().obc_prune_trace(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), steps,
                                           _ptr(order), _ptr(loss), _ptr(w_trace), _ptr(row_status), _ptr(ws), nb,
-                                          _stream(stream)), "obc_prune_trace")
+                                          _opts(opts), _stream(stream)), "obc_prune_trace")
 
 
 def obc_prune_nm(W, Hinv, n_keep, m_block, W_out, row_status, order=None, loss=None, mask=None, row_begin=0,
-                 row_count=None, ws=None, stream=None):
+                 row_count=None, ws=None, opts=None, stream=None):
     """N:M pruning of rows [row_begin, row_begin+row_count): every block of m_block columns keeps n_keep weights."""
     _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(W_out, torch.float32, "W_out")
     _check(row_status, torch.int32, "row_status"); _check(order, torch.int32, "order"); _check(loss, torch.float32, "loss")
@@ -223,11 +236,11 @@ def obc_prune_nm(W, Hinv, n_keep, m_block, W_out, row_status, order=None, loss=N
     ws, nb = _workspace(ws, OP_PRUNE_TRACE, row_count, d, 0, W.device, "obc_prune_nm")
     _raise(load_library().obc_prune_nm(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), int(n_keep),
                                        int(m_block), _ptr(order), _ptr(loss), _ptr(W_out), _ld(W_out), _ptr(mask),
-                                       _ptr(row_status), _ptr(ws), nb, _stream(stream)), "obc_prune_nm")
+                                       _ptr(row_status), _ptr(ws), nb, _opts(opts), _stream(stream)), "obc_prune_nm")
 
 
 def obc_prune_blocks(W, Hinv, order, loss, row_status, block=4, w_trace=None, row_begin=0, row_count=None, ws=None,
-                     stream=None):
+                     opts=None, stream=None):
     """Block pruning (blocks of `block` consecutive columns, Eq. 5) of rows [row_begin, row_begin+row_count): full trace."""
     _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(order, torch.int32, "order")
     _check(loss, torch.float32, "loss"); _check(row_status, torch.int32, "row_status"); _check(w_trace, torch.float32, "w_trace")
@@ -236,7 +249,7 @@ def obc_prune_blocks(W, Hinv, order, loss, row_status, block=4, w_trace=None, ro
     ws, nb = _workspace(ws, OP_PRUNE_BLOCKS, row_count, d, 0, W.device, "obc_prune_blocks")
     _raise(load_library().obc_prune_blocks(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), int(block),
                                            _ptr(order), _ptr(loss), _ptr(w_trace), _ptr(row_status), _ptr(ws), nb,
-                                           _stream(stream)), "obc_prune_blocks")
+                                           _opts(opts), _stream(stream)), "obc_prune_blocks")
 
 
 def obc_select_global_mask(loss, order, k, counts, mask, ws=None, stream=None):
@@ -261,7 +274,7 @@ def obc_select_global_mask_static(loss, order, k, counts, mask, stream=None):
 
 
 def obc_prune_apply(W, Hinv, order, counts, W_out, row_status, w_trace=None, trace_steps=0, row_begin=0,
-                    row_count=None, ws=None, stream=None):
+                    row_count=None, ws=None, opts=None, stream=None):
     """Weights after the first counts[r] eliminations (trace gather if w_trace is given, else replay)."""
     _check(W, torch.float32, "W"); _check(W_out, torch.float32, "W_out"); _check(counts, torch.int32, "counts")
     R, d = W.shape
@@ -273,7 +286,7 @@ def obc_prune_apply(W, Hinv, order, counts, W_out, row_status, w_trace=None, tra
     _raise(load_library().obc_prune_apply(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv),
                                           0 if Hinv is None else _ld(Hinv), _ptr(order), _ptr(counts), _ptr(w_trace),
                                           int(trace_steps), _ptr(W_out), _ld(W_out), _ptr(row_status), _ptr(ws), nb,
-                                          _stream(stream)), "obc_prune_apply")
+                                          _opts(opts), _stream(stream)), "obc_prune_apply")
 
 
 def obc_minmax_grid(W, bits, symmetric, scale, zero, mask=None, stream=None) -> int:
@@ -288,7 +301,7 @@ def obc_minmax_grid(W, bits, symmetric, scale, zero, mask=None, stream=None) -> 
 
 
 def obc_quantize(W, Hinv, scale, zero, bits, symmetric, W_out, codes, row_status, prune_order=None,
-                 prune_counts=None, flags=0, loss=None, qorder=None, row_begin=0, row_count=None, ws=None, stream=None):
+                 prune_counts=None, flags=0, loss=None, qorder=None, row_begin=0, row_count=None, ws=None, opts=None, stream=None):
     """Algorithm 3 (OBQ); with prune_order/prune_counts: replay the pruning first, then quantise survivors."""
     _check(W, torch.float32, "W"); _check(Hinv, torch.float32, "Hinv"); _check(scale, torch.float32, "scale")
     _check(zero, torch.float32, "zero"); _check(W_out, torch.float32, "W_out"); _check(codes, torch.int32, "codes")
@@ -300,4 +313,4 @@ def obc_quantize(W, Hinv, scale, zero, bits, symmetric, W_out, codes, row_status
     _raise(load_library().obc_quantize(_ptr(W), _ld(W), R, d, row_begin, row_count, _ptr(Hinv), _ld(Hinv), _ptr(scale),
                                        _ptr(zero), int(bits), int(bool(symmetric)), _ptr(prune_order), _ptr(prune_counts),
                                        int(flags), _ptr(W_out), _ld(W_out), _ptr(codes), _ptr(loss), _ptr(qorder),
-                                       _ptr(row_status), _ptr(ws), nb, _stream(stream)), "obc_quantize")
+                                       _ptr(row_status), _ptr(ws), nb, _opts(opts), _stream(stream)), "obc_quantize")

@@ -29,10 +29,16 @@ obc_status device_info(DeviceInfo* out) {
     return OBC_OK;
 }
 
-static std::atomic<int> g_engine{OBC_ENGINE_AUTO}, g_engine_threads{0}, g_engine_pending{0};
-int engine_choice() { return g_engine.load(std::memory_order_relaxed); }
-int engine_threads_choice() { return g_engine_threads.load(std::memory_order_relaxed); }
-int engine_pending_choice() { return g_engine_pending.load(std::memory_order_relaxed); }
+// Validates the caller's per-call engine options (NULL = defaults) and copies them.
+static bool engine_opts_ok(const obc_engine_opts* o, EngineOpts* out) {
+    out->engine = OBC_ENGINE_AUTO; out->threads = 0; out->max_pending = 0;
+    if (!o) return true;
+    if (o->engine != OBC_ENGINE_AUTO && o->engine != OBC_ENGINE_STREAMING && o->engine != OBC_ENGINE_BLOCKED) return false;
+    if (o->threads != 0 && o->threads != 128 && o->threads != 256 && o->threads != 512) return false;
+    if (o->max_pending < 0 || o->max_pending > 64 || o->reserved != 0) return false;
+    out->engine = o->engine; out->threads = o->threads; out->max_pending = o->max_pending;
+    return true;
+}
 
 static bool mat_ok(const void* p, int64_t ld, int64_t min_ld) { return p && ld >= min_ld; }
 static bool mat_aligned(const void* p, int64_t ld) { return aligned16(p) && (ld % 4 == 0); }
@@ -64,21 +70,11 @@ const char* obc_status_string(obc_status s) {
 
 unsigned long long obc_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
-obc_status obc_set_engine(obc_engine engine, int threads, int max_pending) {
-    if (engine != OBC_ENGINE_AUTO && engine != OBC_ENGINE_STREAMING && engine != OBC_ENGINE_BLOCKED)
-        return OBC_ERR_INVALID_ARG;
-    if (threads != 0 && threads != 128 && threads != 256 && threads != 512) return OBC_ERR_INVALID_ARG;
-    if (max_pending < 0 || max_pending > 64) return OBC_ERR_INVALID_ARG;
-    g_engine.store((int)engine, std::memory_order_relaxed);
-    g_engine_threads.store(threads, std::memory_order_relaxed);
-    g_engine_pending.store(max_pending, std::memory_order_relaxed);
-    return OBC_OK;
-}
-
-obc_status obc_engine_plan(int d_col, int with_trace, int row_count, int32_t* plan) {
-    if (d_col <= 0 || row_count < 0 || !plan) return OBC_ERR_INVALID_ARG;
-    if (engine_choice() == OBC_ENGINE_STREAMING) return streaming_engine_plan(d_col, plan);
-    return blocked_engine_plan(d_col, with_trace, row_count, plan);
+obc_status obc_engine_plan(int d_col, int with_trace, int row_count, const obc_engine_opts* opts, int32_t* plan) {
+    EngineOpts eo;
+    if (d_col <= 0 || row_count < 0 || !plan || !engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
+    if (eo.engine == OBC_ENGINE_STREAMING) return streaming_engine_plan(d_col, plan);
+    return blocked_engine_plan(d_col, with_trace, row_count, eo, plan);
 }
 
 size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
@@ -148,20 +144,24 @@ obc_status obc_hessian_inverse(const float* H, int d_col, int ldh, float damp_re
 
 obc_status obc_prune_trace(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float* Hinv, int ldhi, int steps, int32_t* order, float* loss, float* w_trace,
-                           int32_t* row_status, void* ws, size_t ws_bytes, obc_stream stream) {
+                           int32_t* row_status, void* ws, size_t ws_bytes, const obc_engine_opts* opts, obc_stream stream) {
+    EngineOpts eo;
+    if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
         return OBC_ERR_INVALID_ARG;
     if (steps < 1 || steps > d_col || !order || !loss || !row_status) return OBC_ERR_INVALID_ARG;
     if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_prune_trace(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, steps, order, loss, w_trace,
-                              row_status, ws, ws_bytes, (cudaStream_t)stream);
+                              row_status, ws, ws_bytes, eo, (cudaStream_t)stream);
 }
 
 obc_status obc_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                         const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
                         float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
-                        obc_stream stream) {
+                        const obc_engine_opts* opts, obc_stream stream) {
+    EngineOpts eo;
+    if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
         return OBC_ERR_INVALID_ARG;
     if (!mat_ok(W_out, ldwo, d_col) || !row_status) return OBC_ERR_INVALID_ARG;
@@ -170,19 +170,21 @@ obc_status obc_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_b
     if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_prune_nm(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, n_keep, m_block, order, loss, W_out,
-                           ldwo, mask, row_status, ws, ws_bytes, (cudaStream_t)stream);
+                           ldwo, mask, row_status, ws, ws_bytes, eo, (cudaStream_t)stream);
 }
 
 obc_status obc_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                             const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
-                            int32_t* row_status, void* ws, size_t ws_bytes, obc_stream stream) {
+                            int32_t* row_status, void* ws, size_t ws_bytes, const obc_engine_opts* opts, obc_stream stream) {
+    EngineOpts eo;
+    if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
         return OBC_ERR_INVALID_ARG;
     if (!order || !loss || !row_status || d_col % 4 != 0) return OBC_ERR_INVALID_ARG;
     if (block != 4 || d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_prune_blocks(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, block, order, loss, w_trace,
-                               row_status, ws, ws_bytes, (cudaStream_t)stream);
+                               row_status, ws, ws_bytes, eo, (cudaStream_t)stream);
 }
 
 obc_status obc_select_global_mask(const float* loss, const int32_t* order, int d_row, int d_col, int64_t k,
@@ -196,7 +198,9 @@ obc_status obc_select_global_mask(const float* loss, const int32_t* order, int d
 obc_status obc_prune_apply(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts,
                            const float* w_trace, int trace_steps, float* W_out, int ldwo, int32_t* row_status,
-                           void* ws, size_t ws_bytes, obc_stream stream) {
+                           void* ws, size_t ws_bytes, const obc_engine_opts* opts, obc_stream stream) {
+    EngineOpts eo;
+    if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !counts || !mat_ok(W_out, ldwo, d_col))
         return OBC_ERR_INVALID_ARG;
     if (w_trace) {
@@ -208,7 +212,7 @@ obc_status obc_prune_apply(const float* W, int ldw, int d_row, int d_col, int ro
     if (d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_replay(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, order, counts, W_out, ldwo,
-                         row_status, ws, ws_bytes, (cudaStream_t)stream);
+                         row_status, ws, ws_bytes, eo, (cudaStream_t)stream);
 }
 
 obc_status obc_minmax_grid(const float* W, int ldw, int d_row, int d_col, const uint8_t* mask, int bits,
@@ -223,7 +227,9 @@ obc_status obc_quantize(const float* W, int ldw, int d_row, int d_col, int row_b
                         const float* Hinv, int ldhi, float* scale, float* zero, int bits, int symmetric,
                         const int32_t* prune_order, const int32_t* prune_counts, int flags, float* W_out, int ldwo,
                         int32_t* codes, float* loss, int32_t* qorder, int32_t* row_status, void* ws,
-                        size_t ws_bytes, obc_stream stream) {
+                        size_t ws_bytes, const obc_engine_opts* opts, obc_stream stream) {
+    EngineOpts eo;
+    if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
         return OBC_ERR_INVALID_ARG;
     if (!scale || !zero || !mat_ok(W_out, ldwo, d_col) || !codes || !row_status) return OBC_ERR_INVALID_ARG;
@@ -234,7 +240,7 @@ obc_status obc_quantize(const float* W, int ldw, int d_row, int d_col, int row_b
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_quantize(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, scale, zero, bits, symmetric,
                            prune_order, prune_counts, flags, W_out, ldwo, codes, loss, qorder, row_status, ws,
-                           ws_bytes, (cudaStream_t)stream);
+                           ws_bytes, eo, (cudaStream_t)stream);
 }
 
 }  // extern "C"

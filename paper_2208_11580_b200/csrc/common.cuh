@@ -56,6 +56,9 @@ __host__ __device__ inline void grid_from_range(float lo, float hi, int bits, in
     }
 }
 
+// The per-call engine options of obc_engine_opts after validation (all zero = defaults).
+struct EngineOpts { int engine; int threads; int max_pending; };
+
 // ---- launchers implemented in the kernel files --------------------------------------------------------------
 size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di);
 size_t select_workspace_bytes(int rows, int d);
@@ -80,22 +83,22 @@ obc_status trace_gather_launch(const float* w_trace, int trace_steps, const int3
                                int row_count, float* W_out, int ldwo, cudaStream_t stream);
 obc_status engine_prune_trace(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                               const float* Hinv, int ldhi, int steps, int32_t* order, float* loss, float* w_trace,
-                              int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream);
+                              int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream);
 obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
                            float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
-                           cudaStream_t stream);
+                           const EngineOpts& eo, cudaStream_t stream);
 obc_status engine_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                                const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
-                               int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream);
+                               int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream);
 size_t engine_blocks_workspace_bytes(int row_count, int d, const DeviceInfo& di);
 obc_status engine_replay(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                          const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts, float* W_out,
-                         int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream);
+                         int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream);
 obc_status engine_quantize(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float* Hinv, int ldhi, float* scale, float* zero, int bits, int symmetric,
                            const int32_t* prune_order, const int32_t* prune_counts, int flags, float* W_out,
                            int ldwo, int32_t* codes, float* loss, int32_t* qorder, int32_t* row_status, void* ws,
-                           size_t ws_bytes, cudaStream_t stream);
+                           size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream);
 
 }  // namespace obc

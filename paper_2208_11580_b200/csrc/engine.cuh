@@ -32,6 +32,7 @@ struct EngineArgs {
     int block_c;                          // blocked engine: 4 = block pruning in blocks of 4 columns (Eq. 5), 0 = off
     float* Gpan; int g_vectors; int g_ld; // blocked engine: overflow pending vectors in global memory (per block
                                           // g_vectors rows of g_ld floats), nullptr = none
+    EngineOpts opts;                      // the caller's per-call choice (host side only)
 };
 
 struct Bcast {                            // block-wide broadcast values, written by one thread
@@ -72,11 +73,7 @@ obc_status streaming_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cuda
 obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream);
 
 obc_status streaming_engine_plan(int d, int32_t* plan);
-obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* plan);
+obc_status blocked_engine_plan(int d, int with_trace, int row_count, const EngineOpts& eo, int32_t* plan);
 
-// Process-wide engine choice (see obc_set_engine in obc.h).
-int engine_choice();
-int engine_threads_choice();
-int engine_pending_choice();
 
 }  // namespace obc

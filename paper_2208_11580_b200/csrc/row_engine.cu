@@ -438,13 +438,14 @@ size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
 }
 
 static obc_status engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
-    if (engine_choice() == OBC_ENGINE_STREAMING) return streaming_engine_launch(a, ws, ws_bytes, stream);
+    if (a.opts.engine == OBC_ENGINE_STREAMING) return streaming_engine_launch(a, ws, ws_bytes, stream);
     return blocked_engine_launch(a, ws, ws_bytes, stream);
 }
 
 static EngineArgs base_args(const float* W, int ldw, int d_col, int row_begin, int row_count, const float* Hinv,
-                            int ldhi, int32_t* row_status) {
+                            int ldhi, int32_t* row_status, const EngineOpts& eo) {
     EngineArgs a = {};
+    a.opts = eo;
     a.W = W; a.ldw = ldw; a.d = d_col; a.row_begin = row_begin; a.row_count = row_count;
     a.Hinv = Hinv; a.ldhi = ldhi; a.row_status = row_status;
     a.bits = 2;
@@ -453,9 +454,9 @@ static EngineArgs base_args(const float* W, int ldw, int d_col, int row_begin, i
 
 obc_status engine_prune_trace(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                               const float* Hinv, int ldhi, int steps, int32_t* order, float* loss, float* w_trace,
-                              int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                              int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream) {
     (void)d_row;
-    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status, eo);
     a.mode = MODE_PRUNE; a.steps = steps; a.order = order; a.loss = loss;
     a.w_trace = w_trace; a.trace_steps = steps;
     return engine_launch(a, ws, ws_bytes, stream);
@@ -464,9 +465,9 @@ obc_status engine_prune_trace(const float* W, int ldw, int d_row, int d_col, int
 obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                            const float* Hinv, int ldhi, int n_keep, int m_block, int32_t* order, float* loss,
                            float* W_out, int ldwo, uint8_t* mask, int32_t* row_status, void* ws, size_t ws_bytes,
-                           cudaStream_t stream) {
+                           const EngineOpts& eo, cudaStream_t stream) {
     (void)d_row;
-    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status, eo);
     a.mode = MODE_PRUNE; a.steps = d_col / m_block * (m_block - n_keep); a.order = order; a.loss = loss;
     a.trace_steps = a.steps; a.W_out = W_out; a.ldwo = ldwo; a.mask = mask;
     a.nm_prune = m_block - n_keep;
@@ -477,9 +478,9 @@ obc_status engine_prune_nm(const float* W, int ldw, int d_row, int d_col, int ro
 
 obc_status engine_prune_blocks(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                                const float* Hinv, int ldhi, int block, int32_t* order, float* loss, float* w_trace,
-                               int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                               int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream) {
     (void)d_row;
-    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status, eo);
     a.mode = MODE_PRUNE; a.steps = d_col; a.order = order; a.loss = loss; a.w_trace = w_trace; a.trace_steps = d_col;
     a.block_c = block;
     return blocked_engine_launch(a, ws, ws_bytes, stream);
@@ -498,9 +499,9 @@ size_t engine_blocks_workspace_bytes(int row_count, int d, const DeviceInfo& di)
 
 obc_status engine_replay(const float* W, int ldw, int d_row, int d_col, int row_begin, int row_count,
                          const float* Hinv, int ldhi, const int32_t* order, const int32_t* counts, float* W_out,
-                         int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                         int ldwo, int32_t* row_status, void* ws, size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream) {
     (void)d_row;
-    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status, eo);
     a.mode = MODE_REPLAY; a.forced_order = order; a.forced_counts = counts; a.W_out = W_out; a.ldwo = ldwo;
     return engine_launch(a, ws, ws_bytes, stream);
 }
@@ -509,9 +510,9 @@ obc_status engine_quantize(const float* W, int ldw, int d_row, int d_col, int ro
                            const float* Hinv, int ldhi, float* scale, float* zero, int bits, int symmetric,
                            const int32_t* prune_order, const int32_t* prune_counts, int flags, float* W_out,
                            int ldwo, int32_t* codes, float* loss, int32_t* qorder, int32_t* row_status, void* ws,
-                           size_t ws_bytes, cudaStream_t stream) {
+                           size_t ws_bytes, const EngineOpts& eo, cudaStream_t stream) {
     (void)d_row;
-    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status);
+    EngineArgs a = base_args(W, ldw, d_col, row_begin, row_count, Hinv, ldhi, row_status, eo);
     a.mode = prune_order ? MODE_REPLAY_QUANT : MODE_QUANT;
     a.forced_order = prune_order; a.forced_counts = prune_counts;
     a.scale = scale; a.zero = zero; a.bits = bits; a.symmetric = symmetric; a.flags = flags;

@@ -1208,9 +1208,9 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 // several of them share an SM; long rows need the shared memory for pending vectors.
 // row_count = rows of the launch (0 = many).
 static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, bool bc = false,
-                     int row_count = 0) {
+                     int row_count = 0, int threads = 0) {
     const int cap = (d + 3) & ~3;
-    int nt = engine_threads_choice();
+    int nt = threads;
     if (nt != 128 && nt != 256 && nt != 512) {
         // measured on full waves of rows: 128 threads win up to d_col ~ 700, 256 up to ~ 1400, 512 above
         nt = d <= 704 ? 128 : (d <= 1408 ? 256 : 512);
@@ -1261,9 +1261,17 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
 }
 
 size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
-    BlkPlan p;
-    if (!blk_plan(d, true, di, &p)) return 256;
-    if (d <= p.ms) return 256;
+    // valid for every per-call choice: a row needs its private triangle whenever d exceeds the on-chip threshold,
+    // and that threshold depends on the threads per row and on the per-row state the call keeps
+    bool off_chip = false;
+    const int nts[4] = {0, 128, 256, 512};
+    for (int k = 0; k < 4; ++k)
+        for (int nm = 0; nm < 2; ++nm) {
+            BlkPlan p;
+            if (!blk_plan(d, true, di, &p, nm != 0, false, row_count, nts[k])) continue;
+            if (d > p.ms) off_chip = true;
+        }
+    if (!off_chip) return 256;
     const int cap = (d + 3) & ~3;
     int blocks = di.sm_count * 4;                 // the largest grid any thread-count choice uses
     if (row_count > 0 && row_count < blocks) blocks = row_count;
@@ -1272,13 +1280,13 @@ size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di
            round_up((size_t)gblocks * BLK_MAXB * ((cap + 15) & ~15) * sizeof(float), 256);
 }
 
-obc_status blocked_engine_plan(int d, int with_trace, int row_count, int32_t* plan) {
+obc_status blocked_engine_plan(int d, int with_trace, int row_count, const EngineOpts& eo, int32_t* plan) {
     DeviceInfo di;
     obc_status st = device_info(&di);
     if (st != OBC_OK) return st;
     BlkPlan p;
-    if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p, false, false, row_count)) return OBC_ERR_UNSUPPORTED;
-    const int mp = engine_pending_choice();
+    if (d > OBC_MAX_DCOL || !blk_plan(d, with_trace != 0, di, &p, false, false, row_count, eo.threads)) return OBC_ERR_UNSUPPORTED;
+    const int mp = eo.max_pending;
     plan[0] = OBC_ENGINE_BLOCKED; plan[1] = p.nt; plan[2] = p.per_sm; plan[3] = p.ms; plan[4] = p.panel_floats;
     plan[5] = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB; plan[6] = di.sm_count; plan[7] = p.g_vectors;
     return OBC_OK;
@@ -1321,10 +1329,10 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     BlkPlan p;
     const bool bc = a.block_c == 4;
-    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc, a.row_count)) return OBC_ERR_UNSUPPORTED;
+    if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc, a.row_count, a.opts.threads)) return OBC_ERR_UNSUPPORTED;
     a.ms = p.ms;
     a.panel_floats = p.panel_floats;
-    int mp = engine_pending_choice();
+    const int mp = a.opts.max_pending;
     a.max_pending = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB;
     if (bc) {
         // groups of 4 slots must stay together: no on-chip tail (it compacts slot by slot), whole blocks per flush

@@ -50,7 +50,7 @@ def prune_layer_sharded(W, X, sparsities, damp_rel: float, prec: int = 2, group=
     """One layer, rows sharded over the ranks of `group` (CUDA tensors, every rank holds all of W and X):
     Hessian and inverse on every rank, pruning trace on the rank's rows, all-gather of the traces, global masks for
     each sparsity on every rank, final weights of the rank's rows.  Returns a dict with the local row range, the
-    global counts/masks per sparsity and the local final weights per sparsity."""
+    global counts/masks per sparsity and the local final weights per sparsity (status: local rows)."""
     import paper_2208_11580_b200 as obc
     world = dist.get_world_size(group) if dist.is_initialized() else 1
     rank = dist.get_rank(group) if dist.is_initialized() else 0
@@ -60,23 +60,28 @@ def prune_layer_sharded(W, X, sparsities, damp_rel: float, prec: int = 2, group=
     H = torch.empty(d, d, dtype=torch.float32, device=dev)
     obc.obc_hessian(X, H, prec=prec)
     Hinv, info = obc.obc_hessian_inverse(H, damp_rel)
-    order = torch.zeros(R, d, dtype=torch.int32, device=dev)
-    loss = torch.zeros(R, d, dtype=torch.float32, device=dev)
-    status = torch.zeros(R, dtype=torch.int32, device=dev)
-    trace = torch.empty(R, d + 1, d, dtype=torch.float32, device=dev) if keep_trace else None
+    # Per-rank buffers hold the LOCAL rows only (the weight trace is count x (d+1) x d, not R x ...): the rank's row
+    # range is handed to the library as a layer of `count` rows of its own, which rows being independent allows.
+    Wl = W[begin:begin + count]
+    order_l = torch.zeros(count, d, dtype=torch.int32, device=dev)
+    loss_l = torch.zeros(count, d, dtype=torch.float32, device=dev)
+    status = torch.zeros(count, dtype=torch.int32, device=dev)
+    trace = torch.empty(count, d + 1, d, dtype=torch.float32, device=dev) if (keep_trace and count) else None
     if count:
-        obc.obc_prune_trace(W, Hinv, order, loss, status, w_trace=trace, row_begin=begin, row_count=count)
+        obc.obc_prune_trace(Wl, Hinv, order_l, loss_l, status, w_trace=trace)
     if world > 1:
-        loss, order = gather_traces(loss[begin:begin + count], order[begin:begin + count], R, group)
+        loss, order = gather_traces(loss_l, order_l, R, group)
+    else:
+        loss, order = loss_l, order_l
     out = {"row_begin": begin, "row_count": count, "info": info, "status": status, "counts": [], "masks": [], "weights": []}
     for sp in sparsities:
         k = int(round(float(sp) * R * d))
         counts = torch.zeros(R, dtype=torch.int32, device=dev)
         mask = torch.zeros(R, d, dtype=torch.uint8, device=dev)
         obc.obc_select_global_mask(loss, order, k, counts, mask)
-        What = torch.zeros(R, d, dtype=torch.float32, device=dev)
+        What = torch.zeros(count, d, dtype=torch.float32, device=dev)
         if count:
-            obc.obc_prune_apply(W, Hinv, order, counts, What, status, w_trace=trace, trace_steps=d if keep_trace else 0,
-                                row_begin=begin, row_count=count)
-        out["counts"].append(counts); out["masks"].append(mask); out["weights"].append(What[begin:begin + count])
+            obc.obc_prune_apply(Wl, Hinv, order_l, counts[begin:begin + count], What, status, w_trace=trace,
+                                trace_steps=d if keep_trace else 0)
+        out["counts"].append(counts); out["masks"].append(mask); out["weights"].append(What)
     return out

@@ -47,11 +47,11 @@ def test_argument_errors_return_before_any_launch(lib):
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(-1.0), good, 8, good, good, 1 << 30, None) == 1
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(0.01), good, 8, None, good, 1 << 30, None) == 1
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(0.01), good, 8, good, good, 64, None) == 3
-    assert lib.obc_prune_trace(good, 8, 4, 8, 2, 3, good, 8, 8, good, good, None, good, good, 1 << 30, None) == 1  # rows
-    assert lib.obc_prune_trace(good, 8, 4, 8, 0, 4, good, 8, 9, good, good, None, good, good, 1 << 30, None) == 1  # steps
-    assert lib.obc_prune_trace(good, 8, 4, 8, 0, 4, good, 8, 8, None, good, None, good, good, 1 << 30, None) == 1
-    assert lib.obc_prune_trace(good, 6000, 4, 6000, 0, 4, good, 6000, 8, good, good, None, good, good, 1 << 30, None) == 8
-    assert lib.obc_prune_trace(good, 10, 4, 8, 0, 4, good, 8, 8, good, good, None, good, good, 1 << 30, None) == 2
+    assert lib.obc_prune_trace(good, 8, 4, 8, 2, 3, good, 8, 8, good, good, None, good, good, 1 << 30, None, None) == 1  # rows
+    assert lib.obc_prune_trace(good, 8, 4, 8, 0, 4, good, 8, 9, good, good, None, good, good, 1 << 30, None, None) == 1  # steps
+    assert lib.obc_prune_trace(good, 8, 4, 8, 0, 4, good, 8, 8, None, good, None, good, good, 1 << 30, None, None) == 1
+    assert lib.obc_prune_trace(good, 6000, 4, 6000, 0, 4, good, 6000, 8, good, good, None, good, good, 1 << 30, None, None) == 8
+    assert lib.obc_prune_trace(good, 10, 4, 8, 0, 4, good, 8, 8, good, good, None, good, good, 1 << 30, None, None) == 2
     assert lib.obc_select_global_mask(good, good, 4, 8, 33, good, good, good, 1 << 30, None) == 1   # k > d_row*d_col
     assert lib.obc_select_global_mask(good, good, 4, 8, -1, good, good, good, 1 << 30, None) == 1
     assert lib.obc_select_global_mask(good, good, 4, 8, 5, good, good, good, 8, None) == 3
@@ -62,11 +62,27 @@ def test_argument_errors_return_before_any_launch(lib):
     assert lib.obc_minmax_grid(good, 8, 4, 8, None, 1, 0, good, good, None, None) == 1              # bits
     assert lib.obc_minmax_grid(good, 8, 4, 8, None, 4, 2, good, good, None, None) == 1              # symmetric flag
     q = lib.obc_quantize
-    assert q(good, 8, 4, 8, 0, 4, good, 8, good, good, 4, 0, good, None, 0, good, 8, good, None, None, good, good, 1 << 30, None) == 1
-    assert q(good, 8, 4, 8, 0, 4, good, 8, good, good, 4, 0, None, None, 4, good, 8, good, None, None, good, good, 1 << 30, None) == 1
-    assert q(good, 8, 4, 8, 0, 4, good, 8, None, good, 4, 0, None, None, 0, good, 8, good, None, None, good, good, 1 << 30, None) == 1
-    assert lib.obc_prune_apply(good, 8, 4, 8, 0, 4, good, 8, good, None, None, 0, good, 8, good, good, 1 << 30, None) == 1
-    assert lib.obc_prune_apply(good, 8, 4, 8, 0, 4, good, 8, good, good, good, 0, good, 8, good, good, 1 << 30, None) == 1
+    assert q(good, 8, 4, 8, 0, 4, good, 8, good, good, 4, 0, good, None, 0, good, 8, good, None, None, good, good, 1 << 30, None, None) == 1
+    assert q(good, 8, 4, 8, 0, 4, good, 8, good, good, 4, 0, None, None, 4, good, 8, good, None, None, good, good, 1 << 30, None, None) == 1
+    assert q(good, 8, 4, 8, 0, 4, good, 8, None, good, 4, 0, None, None, 0, good, 8, good, None, None, good, good, 1 << 30, None, None) == 1
+    assert lib.obc_prune_apply(good, 8, 4, 8, 0, 4, good, 8, good, None, None, 0, good, 8, good, good, 1 << 30, None, None) == 1
+    assert lib.obc_prune_apply(good, 8, 4, 8, 0, 4, good, 8, good, good, good, 0, good, 8, good, good, 1 << 30, None, None) == 1
+
+
+def test_engine_options_are_validated_per_call(lib):
+    """the per-call engine options are checked on the host like every other argument (no process-wide engine state)"""
+    from paper_2208_11580_b200 import binding
+    good = ctypes.c_void_p(0x1000)
+    def trace(opts):
+        return lib.obc_prune_trace(good, 8, 4, 8, 0, 4, good, 8, 8, good, good, None, good, None, 0,
+                                   binding._opts(opts), None)
+    assert trace(binding.EngineOpts(7, 0, 0, 0)) == 1          # unknown engine
+    assert trace(binding.EngineOpts(2, 100, 0, 0)) == 1        # threads not 128/256/512
+    assert trace(binding.EngineOpts(2, 0, 65, 0)) == 1         # more deferred updates than the kernels hold
+    assert trace(binding.EngineOpts(2, 0, 0, 1)) == 1          # reserved field
+    plan = (ctypes.c_int32 * 8)()
+    assert lib.obc_engine_plan(8, 0, 0, binding._opts(binding.EngineOpts(9, 0, 0, 0)), plan) == 1
+    assert "obc_set_engine" not in binding.EXPORTED_SYMBOLS
 
 
 def test_workspace_queries_on_host(lib):

@@ -26,3 +26,19 @@ def test_one_update_per_pass_moves_the_triangle_every_step():
     assert np.isclose(nbytes, 2.0 * d * (d + 1) + float((4.0 * m * (m + 1)).sum()))
     assert np.isclose(flops, float((m * (m + 1)).sum()))
     assert bench.model_bytes_full(4) == 8 * (16 + 9 + 4 + 1)
+
+
+def test_oracle_sample_covers_the_budget_and_scales_by_the_work_model():
+    """the bounded oracle sample of the CPU baseline: whole rows when they fit the budget, else the first eliminations of
+    one row per core, scaled to full rows by sum m^2 (the oracle updates the m x m remaining block at every step)"""
+    rows, steps = bench.oracle_sample(64, 32, 8, 10.0)
+    assert (rows, steps) == (32, 64) and bench.full_row_factor(64, 64) == 1.0
+    rows, steps = bench.oracle_sample(3072, 768, 16, 12.0)
+    assert rows == 16 and 8 <= steps < 3072
+    f = bench.full_row_factor(3072, steps)
+    m = np.arange(1, 3073, dtype=np.float64)
+    assert np.isclose(f, (m ** 2).sum() / (m[-steps:] ** 2).sum()) and f > 1.0
+    # the sampled share of a row's work is about budget / estimated row time
+    est_row = bench.ORACLE_S_PER_UPDATE * (2.0 / 3.0) * 3072 ** 3
+    assert 0.5 < (1.0 / f) / (12.0 / est_row) < 2.0
+    assert bench.full_row_factor(10, 1) == float((np.arange(1, 11) ** 2).sum()) / 100.0

@@ -5,7 +5,7 @@ import torch
 
 import obc_synth
 import oracle
-from parity import check_rows, REL_TOL
+from parity import check_rows, REL_TOL, WithEngineOpts
 
 pytestmark = pytest.mark.gpu
 DAMP = obc_synth.DAMP_REL
@@ -16,9 +16,7 @@ def obc(request):
     """the library with one of its two row elimination engines selected; every test runs with both"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    m.obc_set_engine(m.ENGINE_BLOCKED if request.param == "blocked" else m.ENGINE_STREAMING)
-    yield m
-    m.obc_set_engine(m.ENGINE_AUTO)
+    return WithEngineOpts(m, m.ENGINE_BLOCKED if request.param == "blocked" else m.ENGINE_STREAMING)
 
 
 def dev(a, dtype=None):
@@ -345,32 +343,29 @@ def test_blocked_engine_block_sizes(threads, max_pending, d, rows):
     around the on-chip threshold; prune trace with the full weight trace, and OBQ"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
-    try:
-        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 900 + d, "relu")
-        H = oracle.hessian(X).astype(np.float32)
-        ld = (d + 3) // 4 * 4
-        Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
-        Wd = padded(W, ld)
-        order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
-        assert int(status.abs().sum()) == 0
-        check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
-        scale = torch.zeros(rows, dtype=torch.float32, device="cuda")
-        zero = torch.zeros(rows, dtype=torch.float32, device="cuda")
-        maxq = m.obc_minmax_grid(Wd, 4, False, scale, zero)
-        Wq = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
-        codes = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
-        ql = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
-        qo = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
-        rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
-        m.obc_quantize(Wd, Hinv, scale, zero, 4, False, Wq, codes, rs, loss=ql, qorder=qo)
-        torch.cuda.synchronize()
-        assert int(rs.abs().sum()) == 0
-        check_rows(Hinv.cpu().numpy(), W, qo.cpu().numpy(), ql.cpu().numpy(), gpu_w=Wq.cpu().numpy(), mode="quant",
-                   scale=scale.cpu().numpy().astype(np.float64), zero=zero.cpu().numpy().astype(np.float64), maxq=maxq,
-                   gpu_codes=codes.cpu().numpy())
-    finally:
-        m.obc_set_engine(m.ENGINE_AUTO)
+    m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, max_pending)
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 900 + d, "relu")
+    H = oracle.hessian(X).astype(np.float32)
+    ld = (d + 3) // 4 * 4
+    Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
+    Wd = padded(W, ld)
+    order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
+    assert int(status.abs().sum()) == 0
+    check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
+    scale = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    zero = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    maxq = m.obc_minmax_grid(Wd, 4, False, scale, zero)
+    Wq = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+    codes = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
+    ql = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+    qo = torch.zeros(rows, d, dtype=torch.int32, device="cuda")
+    rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    m.obc_quantize(Wd, Hinv, scale, zero, 4, False, Wq, codes, rs, loss=ql, qorder=qo)
+    torch.cuda.synchronize()
+    assert int(rs.abs().sum()) == 0
+    check_rows(Hinv.cpu().numpy(), W, qo.cpu().numpy(), ql.cpu().numpy(), gpu_w=Wq.cpu().numpy(), mode="quant",
+               scale=scale.cpu().numpy().astype(np.float64), zero=zero.cpu().numpy().astype(np.float64), maxq=maxq,
+               gpu_codes=codes.cpu().numpy())
 
 
 @pytest.mark.parametrize("threads,max_pending,d,rows", [(0, 0, 300, 9), (128, 0, 520, 9), (256, 7, 520, 9), (256, 64, 1100, 6),
@@ -381,45 +376,42 @@ def test_forced_replay_against_trace_and_oracle(threads, max_pending, d, rows):
     the oracle's trace, and -- for an order that names a column twice -- the reported status"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
-    try:
-        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 4100 + d, "relu")
-        H = oracle.hessian(X).astype(np.float32)
-        ld = (d + 3) // 4 * 4
-        Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
-        Wd = padded(W, ld)
-        order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
-        assert int(status.abs().sum()) == 0
-        st = check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
-        cnt = np.array([0, 1, 3, 4, 5, d // 2 + 1, d - 1, d, 37][:rows], dtype=np.int32)
-        counts = torch.from_numpy(cnt).cuda()
-        rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
-        got = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
-        m.obc_prune_apply(Wd, Hinv, order, counts, got, rs)
-        ref = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
-        m.obc_prune_apply(Wd, Hinv, order, counts, ref, rs, w_trace=trace, trace_steps=d)
-        torch.cuda.synchronize()
-        assert int(rs.abs().sum()) == 0
-        g, r = got.cpu().numpy(), ref.cpu().numpy()
-        wscale = np.abs(W).max(axis=1, keepdims=True)
-        assert (np.abs(g - r) / wscale).max() <= REL_TOL
-        want = oracle.weights_from_trace(st["oracle"]["w_trace"], cnt)
-        assert (np.abs(g - want) / wscale).max() <= REL_TOL
-        o = order.cpu().numpy()
-        for i in range(rows):
-            assert np.all(g[i, o[i, :cnt[i]]] == 0.0)
-        # an order that is not a permutation: row 5 names its first column again at step 6
-        bad = order.clone()
-        bad[5, 6] = bad[5, 0]
-        rs2 = torch.zeros(rows, dtype=torch.int32, device="cuda")
-        out2 = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
-        m.obc_prune_apply(Wd, Hinv, bad, counts, out2, rs2)
-        torch.cuda.synchronize()
-        r2 = rs2.cpu().numpy()
-        assert r2[5] == 1 + 6 and np.all(np.delete(r2, 5) == 0)
-        assert np.array_equal(np.delete(out2.cpu().numpy(), 5, axis=0), np.delete(g, 5, axis=0))
-    finally:
-        m.obc_set_engine(m.ENGINE_AUTO)
+    m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, max_pending)
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 4100 + d, "relu")
+    H = oracle.hessian(X).astype(np.float32)
+    ld = (d + 3) // 4 * 4
+    Hinv, info = m.obc_hessian_inverse(padded(H, ld), DAMP)
+    Wd = padded(W, ld)
+    order, loss, status, trace = run_trace(m, Wd, Hinv, want_trace=True)
+    assert int(status.abs().sum()) == 0
+    st = check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy(), gpu_trace=trace.cpu().numpy())
+    cnt = np.array([0, 1, 3, 4, 5, d // 2 + 1, d - 1, d, 37][:rows], dtype=np.int32)
+    counts = torch.from_numpy(cnt).cuda()
+    rs = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    got = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+    m.obc_prune_apply(Wd, Hinv, order, counts, got, rs)
+    ref = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+    m.obc_prune_apply(Wd, Hinv, order, counts, ref, rs, w_trace=trace, trace_steps=d)
+    torch.cuda.synchronize()
+    assert int(rs.abs().sum()) == 0
+    g, r = got.cpu().numpy(), ref.cpu().numpy()
+    wscale = np.abs(W).max(axis=1, keepdims=True)
+    assert (np.abs(g - r) / wscale).max() <= REL_TOL
+    want = oracle.weights_from_trace(st["oracle"]["w_trace"], cnt)
+    assert (np.abs(g - want) / wscale).max() <= REL_TOL
+    o = order.cpu().numpy()
+    for i in range(rows):
+        assert np.all(g[i, o[i, :cnt[i]]] == 0.0)
+    # an order that is not a permutation: row 5 names its first column again at step 6
+    bad = order.clone()
+    bad[5, 6] = bad[5, 0]
+    rs2 = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    out2 = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+    m.obc_prune_apply(Wd, Hinv, bad, counts, out2, rs2)
+    torch.cuda.synchronize()
+    r2 = rs2.cpu().numpy()
+    assert r2[5] == 1 + 6 and np.all(np.delete(r2, 5) == 0)
+    assert np.array_equal(np.delete(out2.cpu().numpy(), 5, axis=0), np.delete(g, 5, axis=0))
 
 
 
@@ -454,29 +446,26 @@ def test_prune_nm_against_oracle(nm, d, rows, threads, max_pending):
     import paper_2208_11580_b200 as m
     m.load_library()
     n_keep, mb = nm
-    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
-    try:
-        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1200 + d + mb, "relu")
-        H = oracle.hessian(X).astype(np.float32)
-        Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
-        Wd = dev(W)
-        steps = d // mb * (mb - n_keep)
-        order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
-        loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
-        Wout = torch.full((rows, d), 9.0, dtype=torch.float32, device="cuda")
-        mask = torch.full((rows, d), 9, dtype=torch.uint8, device="cuda")
-        rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
-        m.obc_prune_nm(Wd, Hinv, n_keep, mb, Wout, rs, order=order, loss=loss, mask=mask)
-        torch.cuda.synchronize()
-        assert int(rs.abs().sum()) == 0
-        o, mk, wo = order.cpu().numpy(), mask.cpu().numpy(), Wout.cpu().numpy()
-        assert np.all(o[:, steps:] == -7) and np.all(mk.reshape(rows, d // mb, mb).sum(axis=2) == n_keep)
-        assert np.all(wo[mk == 0] == 0.0)
-        for r in range(rows):
-            assert set(np.nonzero(mk[r] == 0)[0].tolist()) == set(o[r, :steps].tolist())
-        check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), gpu_w=wo, steps=steps, nm=nm)
-    finally:
-        m.obc_set_engine(m.ENGINE_AUTO)
+    m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, max_pending)
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1200 + d + mb, "relu")
+    H = oracle.hessian(X).astype(np.float32)
+    Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
+    Wd = dev(W)
+    steps = d // mb * (mb - n_keep)
+    order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
+    loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
+    Wout = torch.full((rows, d), 9.0, dtype=torch.float32, device="cuda")
+    mask = torch.full((rows, d), 9, dtype=torch.uint8, device="cuda")
+    rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+    m.obc_prune_nm(Wd, Hinv, n_keep, mb, Wout, rs, order=order, loss=loss, mask=mask)
+    torch.cuda.synchronize()
+    assert int(rs.abs().sum()) == 0
+    o, mk, wo = order.cpu().numpy(), mask.cpu().numpy(), Wout.cpu().numpy()
+    assert np.all(o[:, steps:] == -7) and np.all(mk.reshape(rows, d // mb, mb).sum(axis=2) == n_keep)
+    assert np.all(wo[mk == 0] == 0.0)
+    for r in range(rows):
+        assert set(np.nonzero(mk[r] == 0)[0].tolist()) == set(o[r, :steps].tolist())
+    check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), gpu_w=wo, steps=steps, nm=nm)
 
 
 @pytest.mark.parametrize("threads,max_pending", [(0, 0), (128, 4), (256, 9), (512, 64)])
@@ -486,51 +475,48 @@ def test_prune_blocks_against_oracle(d, rows, kind, threads, max_pending):
     weights after a given number of blocks, and whole-block global masks"""
     import paper_2208_11580_b200 as m
     m.load_library()
-    m.obc_set_engine(m.ENGINE_BLOCKED, threads, max_pending)
-    try:
-        W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1500 + d, kind)
-        H = oracle.hessian(X).astype(np.float32)
-        Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
-        Wd = dev(W)
-        order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
-        loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
-        rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
-        trace = torch.zeros(rows, d + 1, d, dtype=torch.float32, device="cuda")
-        m.obc_prune_blocks(Wd, Hinv, order, loss, rs, w_trace=trace)
-        torch.cuda.synchronize()
-        assert int(rs.abs().sum()) == 0
-        o, l = order.cpu().numpy(), loss.cpu().numpy().astype(np.float64)
-        blocks = o[:, ::4] // 4
-        assert np.array_equal(o, (blocks[:, :, None] * 4 + np.arange(4)).reshape(rows, d))        # members ascending
-        assert all(sorted(blocks[r].tolist()) == list(range(d // 4)) for r in range(rows))
-        assert np.all(l.reshape(rows, d // 4, 4)[:, :, 1:] == 0.0)
-        Hh = Hinv.cpu().numpy().astype(np.float64)
-        res = oracle.run_rows_blocks(Hh, W, 4, forced_blocks=blocks)
-        assert np.all(res["status"] == 0)
-        differ = res["best_block"] != blocks
-        assert not (differ & (res["forced_gap"] > 1e-6)).any()
-        L = res["loss"][:, ::4]
-        floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
-        assert (np.abs(l[:, ::4] - L) / (np.abs(L) + floor)).max() <= REL_TOL
-        assert np.all(trace[:, -1].cpu().numpy() == 0.0)
-        # weights after nb blocks (trace row 4*nb) against the oracle stopped there
-        wscale = np.abs(W).max(axis=1, keepdims=True)
-        for nb in (1, d // 8, d // 4 - 1):
-            part = oracle.run_rows_blocks(Hh, W, 4, steps=nb, forced_blocks=blocks[:, :nb])
-            assert (np.abs(trace[:, 4 * nb].cpu().numpy() - part["w"]) / wscale).max() <= REL_TOL
-        # global step on whole blocks: k a multiple of 4
-        k = (rows * d // 8) * 4
-        counts = torch.zeros(rows, dtype=torch.int32, device="cuda")
-        mask = torch.zeros(rows, d, dtype=torch.uint8, device="cuda")
-        m.obc_select_global_mask(loss, order, k, counts, mask)
-        c, mk = counts.cpu().numpy(), mask.cpu().numpy()
-        assert np.all(c % 4 == 0) and int((mk == 0).sum()) == k
-        per_block = mk.reshape(rows, d // 4, 4).sum(axis=2)
-        assert np.all((per_block == 0) | (per_block == 4))
-        oc, om = oracle.global_mask(l, o, k)
-        assert np.array_equal(c, oc) and np.array_equal(mk, om)
-    finally:
-        m.obc_set_engine(m.ENGINE_AUTO)
+    m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, max_pending)
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1500 + d, kind)
+    H = oracle.hessian(X).astype(np.float32)
+    Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
+    Wd = dev(W)
+    order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
+    loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
+    rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+    trace = torch.zeros(rows, d + 1, d, dtype=torch.float32, device="cuda")
+    m.obc_prune_blocks(Wd, Hinv, order, loss, rs, w_trace=trace)
+    torch.cuda.synchronize()
+    assert int(rs.abs().sum()) == 0
+    o, l = order.cpu().numpy(), loss.cpu().numpy().astype(np.float64)
+    blocks = o[:, ::4] // 4
+    assert np.array_equal(o, (blocks[:, :, None] * 4 + np.arange(4)).reshape(rows, d))        # members ascending
+    assert all(sorted(blocks[r].tolist()) == list(range(d // 4)) for r in range(rows))
+    assert np.all(l.reshape(rows, d // 4, 4)[:, :, 1:] == 0.0)
+    Hh = Hinv.cpu().numpy().astype(np.float64)
+    res = oracle.run_rows_blocks(Hh, W, 4, forced_blocks=blocks)
+    assert np.all(res["status"] == 0)
+    differ = res["best_block"] != blocks
+    assert not (differ & (res["forced_gap"] > 1e-6)).any()
+    L = res["loss"][:, ::4]
+    floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
+    assert (np.abs(l[:, ::4] - L) / (np.abs(L) + floor)).max() <= REL_TOL
+    assert np.all(trace[:, -1].cpu().numpy() == 0.0)
+    # weights after nb blocks (trace row 4*nb) against the oracle stopped there
+    wscale = np.abs(W).max(axis=1, keepdims=True)
+    for nb in (1, d // 8, d // 4 - 1):
+        part = oracle.run_rows_blocks(Hh, W, 4, steps=nb, forced_blocks=blocks[:, :nb])
+        assert (np.abs(trace[:, 4 * nb].cpu().numpy() - part["w"]) / wscale).max() <= REL_TOL
+    # global step on whole blocks: k a multiple of 4
+    k = (rows * d // 8) * 4
+    counts = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    mask = torch.zeros(rows, d, dtype=torch.uint8, device="cuda")
+    m.obc_select_global_mask(loss, order, k, counts, mask)
+    c, mk = counts.cpu().numpy(), mask.cpu().numpy()
+    assert np.all(c % 4 == 0) and int((mk == 0).sum()) == k
+    per_block = mk.reshape(rows, d // 4, 4).sum(axis=2)
+    assert np.all((per_block == 0) | (per_block == 4))
+    oc, om = oracle.global_mask(l, o, k)
+    assert np.array_equal(c, oc) and np.array_equal(mk, om)
 
 
 def test_prune_trace_at_maximum_row_length(obc):
