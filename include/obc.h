@@ -43,7 +43,7 @@ typedef enum {
     OBC_ERR_WORKSPACE = 3,     /* ws is NULL, misaligned or smaller than obc_workspace_bytes(...)        */
     OBC_ERR_NOT_POSDEF = 4,    /* (reported through info[]) Cholesky met a non-positive pivot            */
     OBC_ERR_NONFINITE = 5,     /* (reported through row_status[]) non-positive / non-finite [Hinv]_pp    */
-    OBC_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired                                     */
+    OBC_ERR_TIMEOUT = 6,       /* (reported through info[]) a bounded device-side wait expired           */
     OBC_ERR_CUDA = 7,          /* a CUDA runtime call failed (launch configuration, missing device ...)  */
     OBC_ERR_UNSUPPORTED = 8,   /* size outside what the kernels support (d_col > OBC_MAX_DCOL)           */
     OBC_ERR_STATIC_SCRATCH = 9 /* problem larger than the built-in scratch area of a *_static entry point */
@@ -115,20 +115,29 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n);
  * X: d_col x n, row-major, ldx >= n (one chunk of the calibration axis).  H: d_col x d_col, ldh >= d_col.
  * accumulate = 0 overwrites H, 1 adds to it (Section 3, "Implementation Details": further samples are
  * accumulated into the Hessian once).  H is written in full (both triangles, exactly symmetric).
- * prec picks the tensor-core input precision of the contraction; accumulation is FP32. */
+ * prec picks the tensor-core input precision of the contraction; accumulation is FP32.
+ * The tensor-core kernels synchronise their copy / multiply pipeline through device-side waits, all of them bounded:
+ *   wait_limit : 0 = the built-in bound (about a second per wait); > 0 = that many polls per wait; < 0 = the
+ *                pipeline's waits expire at once (a test hook: it exercises the time-out path without waiting).
+ *   info       : nullable device int32; receives 0, or OBC_ERR_TIMEOUT when a wait expired.  In that case the
+ *                kernel has abandoned its tile cleanly (its copies in flight and issued products are waited for with
+ *                the built-in bound, tensor memory is released), the call has still returned OBC_OK, and H is
+ *                filled with NaN -- also when info is NULL -- so the failure cannot pass unnoticed.
+ * OBC_PREC_FP32 has no waits: wait_limit is ignored and info[0] = 0. */
 obc_status obc_hessian(const float *X, int d_col, int64_t n, int64_t ldx,
-                       float *H, int ldh, int accumulate, obc_prec prec,
+                       float *H, int ldh, int accumulate, obc_prec prec, int32_t *info, int wait_limit,
                        void *ws, size_t ws_bytes, obc_stream stream);
 
 /* Appendix "Sequential Quantization with OBQ": when the layer inputs X come from the already compressed model, the
  * dense weights are first re-fitted in closed form, W^T = (X X^T)^-1 X Y^T (Y = the dense model's outputs, d_row x n),
  * so that they minimise the layer objective again.  X Y^T is accumulated over batches like the Hessian:
  *   obc_cross_gram : G (+)= Y X^T   (G: d_row x d_col, ldg >= d_col; Y: d_row x n, ldy >= n; X: d_col x n, ldx >= n;
- *                    prec as in obc_hessian; workspace obc_workspace_bytes(OBC_OP_CROSS_GRAM, d_row, d_col, n))
+ *                    prec, info, wait_limit as in obc_hessian (G = NaN after a time-out);
+ *                    workspace obc_workspace_bytes(OBC_OP_CROSS_GRAM, d_row, d_col, n))
  *   obc_refit      : W = 2 G Hinv with Hinv = inv(2 X X^T + lambda I) from obc_hessian / obc_hessian_inverse on the
  *                    same X, i.e. the least-squares weights with the solver's dampening lambda/2 on X X^T. */
 obc_status obc_cross_gram(const float *Y, int64_t ldy, const float *X, int64_t ldx, int d_row, int d_col, int64_t n,
-                          float *G, int ldg, int accumulate, obc_prec prec,
+                          float *G, int ldg, int accumulate, obc_prec prec, int32_t *info, int wait_limit,
                           void *ws, size_t ws_bytes, obc_stream stream);
 obc_status obc_refit(const float *G, int ldg, const float *Hinv, int ldhi, int d_row, int d_col,
                      float *W_out, int ldwo, obc_stream stream);

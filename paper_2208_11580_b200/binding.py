@@ -56,9 +56,9 @@ def load_library():
     lib.obc_workspace_bytes.restype = c_sz
     lib.obc_workspace_bytes.argtypes = [c_int, c_int, c_int, c_i64]
     lib.obc_hessian.restype = c_int
-    lib.obc_hessian.argtypes = [vp, c_int, c_i64, c_i64, vp, c_int, c_int, c_int, vp, c_sz, vp]
+    lib.obc_hessian.argtypes = [vp, c_int, c_i64, c_i64, vp, c_int, c_int, c_int, vp, c_int, vp, c_sz, vp]
     lib.obc_cross_gram.restype = c_int
-    lib.obc_cross_gram.argtypes = [vp, c_i64, vp, c_i64, c_int, c_int, c_i64, vp, c_int, c_int, c_int, vp, c_sz, vp]
+    lib.obc_cross_gram.argtypes = [vp, c_i64, vp, c_i64, c_int, c_int, c_i64, vp, c_int, c_int, c_int, vp, c_int, vp, c_sz, vp]
     lib.obc_refit.restype = c_int
     lib.obc_refit.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, c_int, vp]
     lib.obc_hessian_inverse.restype = c_int
@@ -165,17 +165,18 @@ def _raise(status, where):
         raise OBCError(status, where)
 
 
-def obc_hessian(X, H, accumulate=False, prec=PREC_FP32, ws=None, stream=None):
-    """H (+)= 2 X X^T for one chunk X (d_col x n) of the calibration data."""
-    _check(X, torch.float32, "X"); _check(H, torch.float32, "H")
+def obc_hessian(X, H, accumulate=False, prec=PREC_FP32, ws=None, stream=None, info=None, wait_limit=0):
+    """H (+)= 2 X X^T for one chunk X (d_col x n) of the calibration data.  info: optional device int32[1] that
+    receives 0 or the time-out status of the tensor-core kernels' bounded waits (wait_limit: see obc.h)."""
+    _check(X, torch.float32, "X"); _check(H, torch.float32, "H"); _check(info, torch.int32, "info")
     d, n = X.shape
     ws, nb = _workspace(ws, OP_HESSIAN, 0, d, n, X.device, "obc_hessian")
     _raise(load_library().obc_hessian(_ptr(X), d, n, _ld(X), _ptr(H), _ld(H), int(bool(accumulate)), int(prec),
-                                      _ptr(ws), nb, _stream(stream)), "obc_hessian")
+                                      _ptr(info), int(wait_limit), _ptr(ws), nb, _stream(stream)), "obc_hessian")
     return H
 
 
-def obc_cross_gram(Y, X, G, accumulate=False, prec=PREC_FP32, ws=None, stream=None):
+def obc_cross_gram(Y, X, G, accumulate=False, prec=PREC_FP32, ws=None, stream=None, info=None, wait_limit=0):
     """G (+)= Y X^T for one chunk of the calibration axis (Y: d_row x n dense outputs, X: d_col x n inputs)."""
     _check(Y, torch.float32, "Y"); _check(X, torch.float32, "X"); _check(G, torch.float32, "G")
     R, n = Y.shape
@@ -184,7 +185,7 @@ def obc_cross_gram(Y, X, G, accumulate=False, prec=PREC_FP32, ws=None, stream=No
     if prec != PREC_FP32:
         ws, nb = _workspace(ws, OP_CROSS_GRAM, R, d, n, X.device, "obc_cross_gram")
     _raise(load_library().obc_cross_gram(_ptr(Y), _ld(Y), _ptr(X), _ld(X), R, d, n, _ptr(G), _ld(G), int(bool(accumulate)),
-                                         int(prec), _ptr(ws), nb, _stream(stream)), "obc_cross_gram")
+                                         int(prec), _ptr(info), int(wait_limit), _ptr(ws), nb, _stream(stream)), "obc_cross_gram")
     return G
 
 

@@ -101,28 +101,31 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
 }
 
 obc_status obc_hessian(const float* X, int d_col, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
-                       obc_prec prec, void* ws, size_t ws_bytes, obc_stream stream) {
+                       obc_prec prec, int32_t* info, int wait_limit, void* ws, size_t ws_bytes, obc_stream stream) {
     if (d_col <= 0 || n <= 0 || !mat_ok(X, ldx, n) || !mat_ok(H, ldh, d_col)) return OBC_ERR_INVALID_ARG;
     if (accumulate != 0 && accumulate != 1) return OBC_ERR_INVALID_ARG;
     if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
     if (!mat_aligned(X, ldx) || !mat_aligned(H, ldh)) return OBC_ERR_ALIGNMENT;
     if (!ws || !aligned256(ws) || ws_bytes < hessian_workspace_bytes(d_col, n)) return OBC_ERR_WORKSPACE;
-    if (prec == OBC_PREC_FP32) return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, ws, (cudaStream_t)stream);
-    return hessian_tc_launch(X, d_col, n, ldx, H, ldh, accumulate, prec, ws, (cudaStream_t)stream);
+    if (prec == OBC_PREC_FP32) return hessian_fp32_launch(X, d_col, n, ldx, H, ldh, accumulate, info, ws, (cudaStream_t)stream);
+    return hessian_tc_launch(X, d_col, n, ldx, H, ldh, accumulate, prec, info, wait_limit, ws, (cudaStream_t)stream);
 }
 
 obc_status obc_cross_gram(const float* Y, int64_t ldy, const float* X, int64_t ldx, int d_row, int d_col, int64_t n,
-                          float* G, int ldg, int accumulate, obc_prec prec, void* ws, size_t ws_bytes,
-                          obc_stream stream) {
+                          float* G, int ldg, int accumulate, obc_prec prec, int32_t* info, int wait_limit, void* ws,
+                          size_t ws_bytes, obc_stream stream) {
     if (d_row <= 0 || d_col <= 0 || n <= 0 || !mat_ok(Y, ldy, n) || !mat_ok(X, ldx, n) || !mat_ok(G, ldg, d_col))
         return OBC_ERR_INVALID_ARG;
     if (accumulate != 0 && accumulate != 1) return OBC_ERR_INVALID_ARG;
     if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
     if (!mat_aligned(Y, ldy) || !mat_aligned(X, ldx)) return OBC_ERR_ALIGNMENT;
-    if (prec == OBC_PREC_FP32)
+    if (prec == OBC_PREC_FP32) {
+        if (info) OBC_CUDA_TRY(cudaMemsetAsync(info, 0, sizeof(int32_t), (cudaStream_t)stream));   // this path has no waits
         return sgemm_nt_launch(d_row, d_col, n, 1.f, Y, ldy, X, ldx, accumulate ? 1.f : 0.f, G, ldg, (cudaStream_t)stream);
+    }
     if (!ws || !aligned256(ws) || ws_bytes < cross_workspace_bytes(d_row, d_col, n)) return OBC_ERR_WORKSPACE;
-    return cross_tc_launch(Y, d_row, ldy, X, d_col, ldx, n, G, ldg, accumulate, prec, ws, (cudaStream_t)stream);
+    return cross_tc_launch(Y, d_row, ldy, X, d_col, ldx, n, G, ldg, accumulate, prec, info, wait_limit, ws,
+                           (cudaStream_t)stream);
 }
 
 obc_status obc_refit(const float* G, int ldg, const float* Hinv, int ldhi, int d_row, int d_col, float* W_out, int ldwo,

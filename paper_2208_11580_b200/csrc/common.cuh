@@ -69,12 +69,13 @@ obc_status select_launch(const float* loss, const int32_t* order, int rows, int 
 obc_status inverse_launch(const float* H, int d, int ldh, float damp_rel, float* Hinv, int ldhi, int32_t* info,
                           void* ws, cudaStream_t s);
 obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
-                               void* ws, cudaStream_t stream);
+                               int32_t* info, void* ws, cudaStream_t stream);
 obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
-                             obc_prec prec, void* ws, cudaStream_t stream);
+                             obc_prec prec, int32_t* info, int wait_limit, void* ws, cudaStream_t stream);
 size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n);
 obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
-                           float* G, int ldg, int accumulate, obc_prec prec, void* ws, cudaStream_t stream);
+                           float* G, int ldg, int accumulate, obc_prec prec, int32_t* info, int wait_limit, void* ws,
+                           cudaStream_t stream);
 obc_status sgemm_nt_launch(int M, int N, int64_t K, float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                            float beta, float* C, int ldc, cudaStream_t stream);
 obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const uint8_t* mask, int bits, int symmetric,

@@ -101,12 +101,14 @@ __global__ void __launch_bounds__(256) syrk_fp32_kernel(const float* __restrict_
 }
 
 // H[i][j] = H[j][i] = (accumulate ? H[i][j] : 0) + 2 * sum_z partial[z][i][j]     for j <= i
-// err (nullable): a non-zero flag from the producing kernel turns the whole result into NaN.
+// err (nullable): a non-zero flag from the producing kernel (a bounded wait that expired) turns the whole result
+// into NaN; info (nullable) receives 0 or OBC_ERR_TIMEOUT accordingly.
 __global__ void __launch_bounds__(256) hessian_finalize_kernel(const float* __restrict__ partial, int splits, int d,
                                                                float* __restrict__ H, int ldh, int accumulate,
-                                                               const int* __restrict__ err) {
+                                                               const int* __restrict__ err, int32_t* __restrict__ info) {
     const int i = blockIdx.y;
     const int j = blockIdx.x * 256 + threadIdx.x;
+    if (info && i == 0 && j == 0) info[0] = (err && *err != 0) ? (int32_t)OBC_ERR_TIMEOUT : 0;
     if (j > i || j >= d) return;
     float s = 0.f;
     for (int z = 0; z < splits; ++z) s += partial[(size_t)z * d * d + (size_t)i * d + j];
@@ -118,16 +120,16 @@ __global__ void __launch_bounds__(256) hessian_finalize_kernel(const float* __re
 }
 
 obc_status hessian_finalize_launch(const float* partial, int splits, int d, float* H, int ldh, int accumulate,
-                                   const int* err, cudaStream_t stream) {
+                                   const int* err, int32_t* info, cudaStream_t stream) {
     dim3 grid((d + 255) / 256, d);
-    hessian_finalize_kernel<<<grid, 256, 0, stream>>>(partial, splits, d, H, ldh, accumulate, err);
+    hessian_finalize_kernel<<<grid, 256, 0, stream>>>(partial, splits, d, H, ldh, accumulate, err, info);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
 
 obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
-                               void* ws, cudaStream_t stream) {
+                               int32_t* info, void* ws, cudaStream_t stream) {
     const int splits = hessian_splits(d, n);
     int64_t slice = (n + splits - 1) / splits;
     slice = (slice + HK - 1) / HK * HK;
@@ -137,7 +139,7 @@ obc_status hessian_fp32_launch(const float* X, int d, int64_t n, int64_t ldx, fl
     syrk_fp32_kernel<<<grid, 256, 0, stream>>>(X, d, n, ldx, slice, partial);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
-    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, nullptr, stream);
+    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, nullptr, info, stream);
 }
 
 }  // namespace obc

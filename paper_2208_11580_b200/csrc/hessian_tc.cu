@@ -11,9 +11,10 @@
 //   BF16X3  X is first split into hi = bf16(x) and lo = bf16(x - hi); the tile accumulates
 //           hi*hi^T + hi*lo^T + lo*hi^T with kind::f16 (bf16 x bf16), which keeps ~16 mantissa bits.
 //
-// Every wait on an mbarrier is bounded.  If one expires, the CTA raises an error flag, drains its own copies
-// in flight with a bounded wait, frees its tensor memory and returns; the finalize kernel then fills H with
-// NaN so that the failure cannot go unnoticed downstream.
+// Every wait on an mbarrier is bounded (the limit of the pipeline's waits is a kernel argument).  If one expires,
+// the CTA raises an error flag, waits -- with the full built-in limit -- for its own copies in flight and for the
+// products it has issued, frees its tensor memory and returns; the finalize kernel then fills H with NaN and writes
+// OBC_ERR_TIMEOUT to the caller's info word, so that the failure cannot go unnoticed downstream.
 #include "common.cuh"
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -26,11 +27,11 @@ constexpr int TC_TILE = 128;          // output tile (M = N = 128)
 constexpr int TC_KBYTES = 128;        // bytes of K per stage row = one 128B swizzle atom
 constexpr int TC_THREADS = 128;
 constexpr uint32_t TC_TILE_BYTES = TC_TILE * TC_KBYTES;      // 16 KiB per operand tile
-constexpr int TC_WAIT_LIMIT = 4 * 1000 * 1000;
+constexpr int TC_WAIT_LIMIT = 4 * 1000 * 1000;      // polls of a bounded wait (about a second) unless the caller says otherwise
 
 int hessian_splits(int d, int64_t n);
 obc_status hessian_finalize_launch(const float* partial, int splits, int d, float* H, int ldh, int accumulate,
-                                   const int* err, cudaStream_t stream);
+                                   const int* err, int32_t* info, cudaStream_t stream);
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -115,7 +116,7 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
                                                              const __grid_constant__ CUtensorMap map_blo,
                                                              int rows_a, int rows_b, int64_t n_elems, int64_t slice,
                                                              int stages, float* __restrict__ partial,
-                                                             int* __restrict__ err) {
+                                                             int* __restrict__ err, int wait_limit) {
     constexpr int TILES_PER_STAGE = KIND == 0 ? 2 : 4;             // A,B (+ A_lo, B_lo)
     constexpr int KELEMS = KIND == 0 ? 32 : 64;                    // elements of K per stage (128 bytes)
     constexpr int KSTEP = KIND == 0 ? 8 : 16;                      // elements of K per MMA (32 bytes)
@@ -124,6 +125,7 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
     __shared__ __align__(8) unsigned long long bars[2 * 8 + 1];   // full[8], empty[8], accumulator-ready
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ int mma_issued_s;                                   // the issuer has products in flight on the accumulator
 
     int bi = 0, bj = 0;
     if (CROSS) {
@@ -144,6 +146,7 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
         for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         mbar_init(accbar, 1);
         abort_s = 0;
+        mma_issued_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {                                               // one warp allocates the accumulator columns
@@ -161,7 +164,7 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
         // ---- TMA producer ---------------------------------------------------------------------------------
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % stages;
-            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, TC_WAIT_LIMIT)) {
+            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, wait_limit)) {
                 atomicExch(err, 1); abort_s = 1; break;
             }
             if (*(volatile int*)&abort_s) break;
@@ -181,9 +184,10 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
         const uint32_t idesc = instr_desc(KIND == 0 ? 2u : 1u);
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % stages;
-            if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, TC_WAIT_LIMIT)) { atomicExch(err, 2); abort_s = 1; break; }
+            if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, wait_limit)) { atomicExch(err, 2); abort_s = 1; break; }
             if (*(volatile int*)&abort_s) break;
             tc_fence_after();
+            mma_issued_s = 1;
             const uint32_t base = smem_u32(tiles) + s * stage_bytes;
             const uint64_t da = smem_desc_sw128(base), db = smem_desc_sw128(base + TC_TILE_BYTES);
 #pragma unroll
@@ -201,13 +205,14 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
             }
             tc_commit(empty0 + 8 * s);                             // frees the stage when these MMAs have read it
         }
-        tc_commit(accbar);                                         // accumulator complete
+        // accumulator complete (after an abort: completion of whatever was issued, which the exit path waits for)
+        if (nkb > 0 && *(volatile int*)&mma_issued_s) tc_commit(accbar);
     }
     __syncwarp();
     // ---- epilogue: all four warps, warp w owns accumulator lanes 32w .. 32w+31 ------------------------------------
     bool ok = true;
     if (nkb > 0) {
-        if (lane == 0) ok = mbar_wait(accbar, 0, TC_WAIT_LIMIT);
+        if (lane == 0) ok = mbar_wait(accbar, 0, wait_limit);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok && lane == 0) { atomicExch(err, 3); abort_s = 1; }
     }
@@ -236,9 +241,12 @@ __global__ void __launch_bounds__(TC_THREADS) syrk_tc_kernel(const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (*(volatile int*)&abort_s && warp == 0 && lane == 0) {
-        // drain our own copies in flight (bounded) so that nothing lands in shared memory after we exit
+        // Wait, with the full limit whatever the caller's, for our own copies in flight, so that nothing lands in
+        // shared memory after we exit, and for the products issued so far, so that tensor memory is idle when it is
+        // freed.  (Only the youngest phase of a stage can still be pending; older ones were consumed before reuse.)
         for (int kb = issued > stages ? issued - stages : 0; kb < issued; ++kb)
             mbar_wait(full0 + 8 * (kb % stages), (kb / stages) & 1, TC_WAIT_LIMIT);
+        if (*(volatile int*)&mma_issued_s) mbar_wait(accbar, 0, TC_WAIT_LIMIT);
     }
     __syncthreads();
     if (warp == 0) {
@@ -307,8 +315,12 @@ size_t hessian_tc_extra_bytes(int d, int64_t n) {          // error flag + bf16 
     return 256 + 2 * round_up((size_t)d * n_pad * sizeof(__nv_bfloat16), 256);
 }
 
+// wait_limit: 0 = the built-in limit, > 0 = that many polls, < 0 = the pipeline's waits expire at once.
+static int resolve_wait_limit(int wait_limit) { return wait_limit == 0 ? TC_WAIT_LIMIT : (wait_limit < 0 ? 0 : wait_limit); }
+
 obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, float* H, int ldh, int accumulate,
-                             obc_prec prec, void* ws, cudaStream_t stream) {
+                             obc_prec prec, int32_t* info, int wait_limit, void* ws, cudaStream_t stream) {
+    const int wl = resolve_wait_limit(wait_limit);
     const int splits = hessian_splits(d, n);
     char* p = reinterpret_cast<char*>(ws);
     float* partial = reinterpret_cast<float*>(p); p += round_up((size_t)splits * d * d * sizeof(float), 256);
@@ -328,7 +340,7 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
         const int stages = 6;
         const size_t smem = (size_t)stages * 2 * TC_TILE_BYTES + 1024;
         OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<0, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n, slice, stages, partial, err);
+        syrk_tc_kernel<0, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n, slice, stages, partial, err, wl);
         count_launch();
     } else {
         split_bf16_kernel<<<1184, 256, 0, stream>>>(X, d, n, ldx, n_pad, hi, lo);
@@ -338,11 +350,11 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
         const int stages = 3;
         const size_t smem = (size_t)stages * 4 * TC_TILE_BYTES + 1024;
         OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<1, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n_pad, slice, stages, partial, err);
+        syrk_tc_kernel<1, false><<<grid, TC_THREADS, smem, stream>>>(ma, ml, ma, ml, d, d, n_pad, slice, stages, partial, err, wl);
         count_launch();
     }
     OBC_CUDA_TRY(cudaGetLastError());
-    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, err, stream);
+    return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, err, info, stream);
 }
 
 // ---- G (+)= Y X^T on the tensor cores (appendix "Sequential Quantization with OBQ": X Y^T is accumulated over
@@ -367,9 +379,10 @@ size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n) {
 
 __global__ void __launch_bounds__(256) cross_finalize_kernel(const float* __restrict__ partial, int splits, int rows_a,
                                                              int rows_b, float* __restrict__ G, int ldg, int accumulate,
-                                                             const int* __restrict__ err) {
+                                                             const int* __restrict__ err, int32_t* __restrict__ info) {
     const int i = blockIdx.y;
     const int j = blockIdx.x * 256 + threadIdx.x;
+    if (info && i == 0 && j == 0) info[0] = (err && *err != 0) ? (int32_t)OBC_ERR_TIMEOUT : 0;
     if (j >= rows_b) return;
     float s = 0.f;
     for (int z = 0; z < splits; ++z) s += partial[(size_t)z * rows_a * rows_b + (size_t)i * rows_b + j];
@@ -379,7 +392,9 @@ __global__ void __launch_bounds__(256) cross_finalize_kernel(const float* __rest
 }
 
 obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
-                           float* G, int ldg, int accumulate, obc_prec prec, void* ws, cudaStream_t stream) {
+                           float* G, int ldg, int accumulate, obc_prec prec, int32_t* info, int wait_limit, void* ws,
+                           cudaStream_t stream) {
+    const int wl = resolve_wait_limit(wait_limit);
     const int splits = cross_splits(rows_a, rows_b, n);
     char* p = reinterpret_cast<char*>(ws);
     float* partial = reinterpret_cast<float*>(p); p += round_up((size_t)splits * rows_a * rows_b * sizeof(float), 256);
@@ -402,7 +417,7 @@ obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float*
         const int stages = 6;
         const size_t smem = (size_t)stages * 2 * TC_TILE_BYTES + 1024;
         OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<0, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n, slice, stages, partial, err);
+        syrk_tc_kernel<0, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n, slice, stages, partial, err, wl);
         count_launch();
     } else {
         split_bf16_kernel<<<1184, 256, 0, stream>>>(Y, rows_a, n, ldy, n_pad, yhi, ylo);
@@ -415,12 +430,12 @@ obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float*
         const int stages = 3;
         const size_t smem = (size_t)stages * 4 * TC_TILE_BYTES + 1024;
         OBC_CUDA_TRY(cudaFuncSetAttribute(syrk_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        syrk_tc_kernel<1, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n_pad, slice, stages, partial, err);
+        syrk_tc_kernel<1, true><<<grid, TC_THREADS, smem, stream>>>(ma, mal, mb, mbl, rows_a, rows_b, n_pad, slice, stages, partial, err, wl);
         count_launch();
     }
     OBC_CUDA_TRY(cudaGetLastError());
     dim3 fgrid((rows_b + 255) / 256, rows_a);
-    cross_finalize_kernel<<<fgrid, 256, 0, stream>>>(partial, splits, rows_a, rows_b, G, ldg, accumulate, err);
+    cross_finalize_kernel<<<fgrid, 256, 0, stream>>>(partial, splits, rows_a, rows_b, G, ldg, accumulate, err, info);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;

@@ -14,7 +14,9 @@ import numpy as np
 import oracle
 
 MARGIN_TOL = 1e-6      # picks must agree wherever best and forced scores differ by more than this (relative)
-REL_TOL = 1e-4         # loss traces and weights: relative error bound in FP32
+REL_TOL = 1e-4         # loss traces and weights: relative error bound in FP32.  Weights are compared relative to
+                       # max(|reference entry|, largest initial weight of the row): late in a row the few remaining
+                       # weights carry the compensation of all the others and grow to several times the initial scale
 ROUND_TOL = 1e-4       # integer codes may differ only if x/Delta is this close to a rounding boundary
 
 
@@ -85,19 +87,22 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
             stats["codes_differ"] = int(cd.sum())
             assert not (cd & (rd_by_col > ROUND_TOL)).any(), "integer codes differ away from rounding boundaries"
             same = ~cd
-            werr = np.abs(gw - res["w"]) / wscale
+            werr = np.abs(gw - res["w"]) / np.maximum(np.abs(res["w"]), wscale)
             stats["w_max_rel"] = float(werr[same].max()) if same.any() else 0.0
             assert werr[same].max() <= REL_TOL
         else:
-            werr = np.abs(gw - res["w"]) / wscale
+            werr = np.abs(gw - res["w"]) / np.maximum(np.abs(res["w"]), wscale)
             stats["w_max_rel"] = float(werr.max())
             assert werr.max() <= REL_TOL, f"weights off by {werr.max():.3e}"
     if gpu_trace is not None:
         gt = np.asarray(gpu_trace, dtype=np.float64)
         wscale = np.abs(W).max(axis=1)[:, None, None]
-        terr = np.abs(gt - res["w_trace"]) / wscale
+        terr = np.abs(gt - res["w_trace"]) / np.maximum(np.abs(res["w_trace"]), wscale)
         stats["trace_max_rel"] = float(terr.max())
-        assert terr.max() <= REL_TOL
+        stats["trace_max_over_initial_scale"] = float((np.abs(gt - res["w_trace"]) / wscale).max())
+        stats["trace_rows_max_rel"] = [float(x) for x in terr.reshape(rows, -1).max(axis=1)]
+        assert terr.max() <= REL_TOL, (f"weight trace off by {terr.max():.3e} at (row, step, column) "
+                                       f"{np.unravel_index(terr.argmax(), terr.shape)}; per row {stats['trace_rows_max_rel']}")
     stats["oracle"] = res
     return stats
 

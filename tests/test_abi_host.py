@@ -36,14 +36,14 @@ def test_argument_errors_return_before_any_launch(lib):
     f = ctypes.c_void_p
     good = f(0x1000)
     # NULL / negative / inconsistent sizes
-    assert lib.obc_hessian(None, 8, 16, 16, good, 8, 0, 0, good, 1 << 30, None) == 1
-    assert lib.obc_hessian(good, 8, 16, 8, good, 8, 0, 0, good, 1 << 30, None) == 1       # ldx < n
-    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 2, 0, good, 1 << 30, None) == 1       # accumulate flag
-    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 9, good, 1 << 30, None) == 1       # precision enum
-    assert lib.obc_hessian(f(0x1004), 8, 16, 16, good, 8, 0, 0, good, 1 << 30, None) == 2  # misaligned X
-    assert lib.obc_hessian(good, 8, 16, 18, good, 8, 0, 0, good, 1 << 30, None) == 2       # ldx % 4
-    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 0, None, 0, None) == 3             # no workspace
-    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 0, good, 16, None) == 3            # too small
+    assert lib.obc_hessian(None, 8, 16, 16, good, 8, 0, 0, None, 0, good, 1 << 30, None) == 1
+    assert lib.obc_hessian(good, 8, 16, 8, good, 8, 0, 0, None, 0, good, 1 << 30, None) == 1       # ldx < n
+    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 2, 0, None, 0, good, 1 << 30, None) == 1       # accumulate flag
+    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 9, None, 0, good, 1 << 30, None) == 1       # precision enum
+    assert lib.obc_hessian(f(0x1004), 8, 16, 16, good, 8, 0, 0, None, 0, good, 1 << 30, None) == 2  # misaligned X
+    assert lib.obc_hessian(good, 8, 16, 18, good, 8, 0, 0, None, 0, good, 1 << 30, None) == 2       # ldx % 4
+    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 0, None, 0, None, 0, None) == 3    # no workspace
+    assert lib.obc_hessian(good, 8, 16, 16, good, 8, 0, 0, None, 0, good, 16, None) == 3   # too small
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(-1.0), good, 8, good, good, 1 << 30, None) == 1
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(0.01), good, 8, None, good, 1 << 30, None) == 1
     assert lib.obc_hessian_inverse(good, 8, 8, ctypes.c_float(0.01), good, 8, good, good, 64, None) == 3
