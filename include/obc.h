@@ -58,7 +58,7 @@ enum {
 
 typedef enum {
     OBC_OP_HESSIAN = 0, OBC_OP_INVERSE = 1, OBC_OP_PRUNE_TRACE = 2, OBC_OP_SELECT = 3,
-    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5, OBC_OP_PRUNE_BLOCKS = 6, OBC_OP_CROSS_GRAM = 7
+    OBC_OP_PRUNE_APPLY = 4, OBC_OP_QUANTIZE = 5, OBC_OP_PRUNE_BLOCKS = 6, OBC_OP_CROSS_GRAM = 7, OBC_OP_REFIT = 8
 } obc_op;
 
 /* Which row elimination engine obc_prune_trace / obc_prune_apply / obc_quantize run (all compute Algorithm 1 /
@@ -85,15 +85,19 @@ unsigned long long obc_kernel_launches(void);
  *   threads     : BLOCKED engine, threads per row: 128, 256, 512, or 0 = chosen from d_col and row_count.
  *   max_pending : BLOCKED engine, upper limit on the number of deferred updates, 1..64, or 0 = as many as the
  *                 shared memory holds.
- *   reserved    : must be 0.
+ *   flags       : OBC_ENGINE_WHOLE_WAVES or 0.  By default, when a call has more rows than the GPU holds at once and
+ *                 they do not divide evenly, the BLOCKED engine gives every thread block the same amount of work, so a
+ *                 row may be started by one block and finished by another; with OBC_ENGINE_WHOLE_WAVES every row stays
+ *                 on one block and the last wave runs partly empty.
  * Values outside these sets make the call return OBC_ERR_INVALID_ARG.  Workspace sizes reported by
  * obc_workspace_bytes are valid for every choice. */
 typedef struct {
     int32_t engine;
     int32_t threads;
     int32_t max_pending;
-    int32_t reserved;
+    int32_t flags;
 } obc_engine_opts;
+enum { OBC_ENGINE_WHOLE_WAVES = 1 };
 
 /* How the row engines would run row_count rows (0 = many) of length d_col on the CURRENT device with the options
  * `opts` (host function, no launch).  with_trace != 0: as for obc_prune_trace with a weight trace.
@@ -135,12 +139,15 @@ obc_status obc_hessian(const float *X, int d_col, int64_t n, int64_t ldx,
  *                    prec, info, wait_limit as in obc_hessian (G = NaN after a time-out);
  *                    workspace obc_workspace_bytes(OBC_OP_CROSS_GRAM, d_row, d_col, n))
  *   obc_refit      : W = 2 G Hinv with Hinv = inv(2 X X^T + lambda I) from obc_hessian / obc_hessian_inverse on the
- *                    same X, i.e. the least-squares weights with the solver's dampening lambda/2 on X X^T. */
+ *                    same X, i.e. the least-squares weights with the solver's dampening lambda/2 on X X^T.  A dense
+ *                    d_row x d_col x d_col contraction: prec = OBC_PREC_FP32 runs it on the CUDA cores (no workspace),
+ *                    TF32 / BF16X3 on the tensor cores with the kernel of obc_cross_gram (workspace
+ *                    obc_workspace_bytes(OBC_OP_REFIT, d_row, d_col, 0); a time-out of its bounded waits leaves NaN). */
 obc_status obc_cross_gram(const float *Y, int64_t ldy, const float *X, int64_t ldx, int d_row, int d_col, int64_t n,
                           float *G, int ldg, int accumulate, obc_prec prec, int32_t *info, int wait_limit,
                           void *ws, size_t ws_bytes, obc_stream stream);
 obc_status obc_refit(const float *G, int ldg, const float *Hinv, int ldhi, int d_row, int d_col,
-                     float *W_out, int ldwo, obc_stream stream);
+                     float *W_out, int ldwo, obc_prec prec, void *ws, size_t ws_bytes, obc_stream stream);
 
 /* Section 3 ("Implementation Details"): Hinv = inv(H + damp_rel * mean(diag H) * I) through a Cholesky
  * factorisation carried in FP64, written as an exactly symmetric FP32 matrix (ldhi >= d_col).

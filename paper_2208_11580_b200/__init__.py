@@ -7,7 +7,7 @@ ABI.  There is no CPU or PyTorch fallback: calling any function without the buil
 from .binding import (  # noqa: F401
     OBCError, library_path, load_library, obc_hessian, obc_cross_gram, obc_refit, obc_hessian_inverse, obc_minmax_grid, obc_prune_apply,
     obc_prune_trace, obc_prune_nm, obc_prune_blocks, obc_quantize, obc_select_global_mask, obc_select_global_mask_static, obc_status_string, obc_workspace_bytes, obc_kernel_launches,
-    obc_engine_plan, EngineOpts, engine_opts, ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED,
-    OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS, OP_CROSS_GRAM,
+    obc_engine_plan, EngineOpts, engine_opts, ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED, ENGINE_WHOLE_WAVES,
+    OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS, OP_CROSS_GRAM, OP_REFIT,
     PREC_FP32, PREC_TF32, PREC_BF16X3, FLAG_OUTLIERS, EXPORTED_SYMBOLS,
 )

@@ -13,10 +13,11 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIBPATH = os.path.join(_HERE, "libobc.so")
 
-OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS, OP_CROSS_GRAM = range(8)
+OP_HESSIAN, OP_INVERSE, OP_PRUNE_TRACE, OP_SELECT, OP_PRUNE_APPLY, OP_QUANTIZE, OP_PRUNE_BLOCKS, OP_CROSS_GRAM, OP_REFIT = range(9)
 PREC_FP32, PREC_TF32, PREC_BF16X3 = 0, 1, 2
 FLAG_OUTLIERS = 1
 ENGINE_AUTO, ENGINE_STREAMING, ENGINE_BLOCKED = 0, 1, 2
+ENGINE_WHOLE_WAVES = 1
 
 EXPORTED_SYMBOLS = (
     "obc_status_string", "obc_kernel_launches", "obc_engine_plan", "obc_workspace_bytes", "obc_hessian", "obc_cross_gram", "obc_refit", "obc_hessian_inverse", "obc_prune_trace", "obc_prune_nm", "obc_prune_blocks",
@@ -60,7 +61,7 @@ def load_library():
     lib.obc_cross_gram.restype = c_int
     lib.obc_cross_gram.argtypes = [vp, c_i64, vp, c_i64, c_int, c_int, c_i64, vp, c_int, c_int, c_int, vp, c_int, vp, c_sz, vp]
     lib.obc_refit.restype = c_int
-    lib.obc_refit.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, c_int, vp]
+    lib.obc_refit.argtypes = [vp, c_int, vp, c_int, c_int, c_int, vp, c_int, c_int, vp, c_sz, vp]
     lib.obc_hessian_inverse.restype = c_int
     lib.obc_hessian_inverse.argtypes = [vp, c_int, c_int, c_f, vp, c_int, vp, vp, c_sz, vp]
     lib.obc_prune_trace.restype = c_int
@@ -98,11 +99,11 @@ class EngineOpts(ctypes.Structure):
     """obc_engine_opts: per-call choice of the row elimination engine (engine, threads per row, limit on deferred
     updates); all zero = the library's defaults."""
     _fields_ = [("engine", ctypes.c_int32), ("threads", ctypes.c_int32), ("max_pending", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("flags", ctypes.c_int32)]
 
 
-def engine_opts(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0) -> EngineOpts:
-    return EngineOpts(int(engine), int(threads), int(max_pending), 0)
+def engine_opts(engine: int = ENGINE_AUTO, threads: int = 0, max_pending: int = 0, flags: int = 0) -> EngineOpts:
+    return EngineOpts(int(engine), int(threads), int(max_pending), int(flags))
 
 
 def _opts(opts):
@@ -189,12 +190,16 @@ def obc_cross_gram(Y, X, G, accumulate=False, prec=PREC_FP32, ws=None, stream=No
     return G
 
 
-def obc_refit(G, Hinv, W_out, stream=None):
-    """W_out = 2 G Hinv: the dense least-squares weights for the inputs behind G and Hinv."""
+def obc_refit(G, Hinv, W_out, prec=PREC_FP32, ws=None, stream=None):
+    """W_out = 2 G Hinv: the dense least-squares weights for the inputs behind G and Hinv (prec: CUDA cores or the
+    tensor-core kernel of obc_cross_gram)."""
     _check(G, torch.float32, "G"); _check(Hinv, torch.float32, "Hinv"); _check(W_out, torch.float32, "W_out")
     R, d = G.shape
-    _raise(load_library().obc_refit(_ptr(G), _ld(G), _ptr(Hinv), _ld(Hinv), R, d, _ptr(W_out), _ld(W_out),
-                                    _stream(stream)), "obc_refit")
+    nb = 0
+    if prec != PREC_FP32:
+        ws, nb = _workspace(ws, OP_REFIT, R, d, 0, G.device, "obc_refit")
+    _raise(load_library().obc_refit(_ptr(G), _ld(G), _ptr(Hinv), _ld(Hinv), R, d, _ptr(W_out), _ld(W_out), int(prec),
+                                    _ptr(ws), nb, _stream(stream)), "obc_refit")
     return W_out
 
 

@@ -31,12 +31,12 @@ obc_status device_info(DeviceInfo* out) {
 
 // Validates the caller's per-call engine options (NULL = defaults) and copies them.
 static bool engine_opts_ok(const obc_engine_opts* o, EngineOpts* out) {
-    out->engine = OBC_ENGINE_AUTO; out->threads = 0; out->max_pending = 0;
+    out->engine = OBC_ENGINE_AUTO; out->threads = 0; out->max_pending = 0; out->flags = 0;
     if (!o) return true;
     if (o->engine != OBC_ENGINE_AUTO && o->engine != OBC_ENGINE_STREAMING && o->engine != OBC_ENGINE_BLOCKED) return false;
     if (o->threads != 0 && o->threads != 128 && o->threads != 256 && o->threads != 512) return false;
-    if (o->max_pending < 0 || o->max_pending > 64 || o->reserved != 0) return false;
-    out->engine = o->engine; out->threads = o->threads; out->max_pending = o->max_pending;
+    if (o->max_pending < 0 || o->max_pending > 64 || (o->flags & ~OBC_ENGINE_WHOLE_WAVES)) return false;
+    out->engine = o->engine; out->threads = o->threads; out->max_pending = o->max_pending; out->flags = o->flags;
     return true;
 }
 
@@ -84,6 +84,7 @@ size_t obc_workspace_bytes(obc_op op, int row_count, int d_col, int64_t n) {
         case OBC_OP_INVERSE: return inverse_workspace_bytes(d_col);
         case OBC_OP_SELECT: return row_count > 0 ? select_workspace_bytes(row_count, d_col) : 0;
         case OBC_OP_CROSS_GRAM: return (n > 0 && row_count > 0) ? cross_workspace_bytes(row_count, d_col, n) : 0;
+        case OBC_OP_REFIT: return row_count > 0 ? cross_workspace_bytes(row_count, d_col, d_col) : 0;
         case OBC_OP_PRUNE_BLOCKS: {
             DeviceInfo di;
             if (device_info(&di) != OBC_OK || d_col > OBC_MAX_DCOL) return 0;
@@ -124,16 +125,22 @@ obc_status obc_cross_gram(const float* Y, int64_t ldy, const float* X, int64_t l
         return sgemm_nt_launch(d_row, d_col, n, 1.f, Y, ldy, X, ldx, accumulate ? 1.f : 0.f, G, ldg, (cudaStream_t)stream);
     }
     if (!ws || !aligned256(ws) || ws_bytes < cross_workspace_bytes(d_row, d_col, n)) return OBC_ERR_WORKSPACE;
-    return cross_tc_launch(Y, d_row, ldy, X, d_col, ldx, n, G, ldg, accumulate, prec, info, wait_limit, ws,
+    return cross_tc_launch(Y, d_row, ldy, X, d_col, ldx, n, G, ldg, accumulate, 1.f, prec, info, wait_limit, ws,
                            (cudaStream_t)stream);
 }
 
 obc_status obc_refit(const float* G, int ldg, const float* Hinv, int ldhi, int d_row, int d_col, float* W_out, int ldwo,
-                     obc_stream stream) {
+                     obc_prec prec, void* ws, size_t ws_bytes, obc_stream stream) {
     if (d_row <= 0 || d_col <= 0 || !mat_ok(G, ldg, d_col) || !mat_ok(Hinv, ldhi, d_col) || !mat_ok(W_out, ldwo, d_col))
         return OBC_ERR_INVALID_ARG;
-    // Hinv is symmetric, so G Hinv = G Hinv^T is the "A B^T" product
-    return sgemm_nt_launch(d_row, d_col, d_col, 2.f, G, ldg, Hinv, ldhi, 0.f, W_out, ldwo, (cudaStream_t)stream);
+    if (prec != OBC_PREC_FP32 && prec != OBC_PREC_TF32 && prec != OBC_PREC_BF16X3) return OBC_ERR_INVALID_ARG;
+    // Hinv is symmetric, so G Hinv = G Hinv^T is the "A B^T" product (contraction over d_col)
+    if (prec == OBC_PREC_FP32)
+        return sgemm_nt_launch(d_row, d_col, d_col, 2.f, G, ldg, Hinv, ldhi, 0.f, W_out, ldwo, (cudaStream_t)stream);
+    if (!mat_aligned(G, ldg) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
+    if (!ws || !aligned256(ws) || ws_bytes < cross_workspace_bytes(d_row, d_col, d_col)) return OBC_ERR_WORKSPACE;
+    return cross_tc_launch(G, d_row, ldg, Hinv, d_col, ldhi, d_col, W_out, ldwo, 0, 2.f, prec, nullptr, 0, ws,
+                           (cudaStream_t)stream);
 }
 
 obc_status obc_hessian_inverse(const float* H, int d_col, int ldh, float damp_rel, float* Hinv, int ldhi,

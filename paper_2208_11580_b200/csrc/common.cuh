@@ -57,7 +57,7 @@ __host__ __device__ inline void grid_from_range(float lo, float hi, int bits, in
 }
 
 // The per-call engine options of obc_engine_opts after validation (all zero = defaults).
-struct EngineOpts { int engine; int threads; int max_pending; };
+struct EngineOpts { int engine; int threads; int max_pending; int flags; };
 
 // ---- launchers implemented in the kernel files --------------------------------------------------------------
 size_t engine_workspace_bytes(int row_count, int d, const DeviceInfo& di);
@@ -74,8 +74,8 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
                              obc_prec prec, int32_t* info, int wait_limit, void* ws, cudaStream_t stream);
 size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n);
 obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
-                           float* G, int ldg, int accumulate, obc_prec prec, int32_t* info, int wait_limit, void* ws,
-                           cudaStream_t stream);
+                           float* G, int ldg, int accumulate, float alpha, obc_prec prec, int32_t* info, int wait_limit,
+                           void* ws, cudaStream_t stream);
 obc_status sgemm_nt_launch(int M, int N, int64_t K, float alpha, const float* A, int64_t lda, const float* B, int64_t ldb,
                            float beta, float* C, int ldc, cudaStream_t stream);
 obc_status minmax_grid_launch(const float* W, int ldw, int rows, int d, const uint8_t* mask, int bits, int symmetric,

@@ -32,6 +32,10 @@ struct EngineArgs {
     int block_c;                          // blocked engine: 4 = block pruning in blocks of 4 columns (Eq. 5), 0 = off
     float* Gpan; int g_vectors; int g_ld; // blocked engine: overflow pending vectors in global memory (per block
                                           // g_vectors rows of g_ld floats), nullptr = none
+    int split;                            // blocked engine: rows are shared out in equal work per block, a row may be
+                                          // started by one block and finished by the next (see row_engine_blocked.cu)
+    char* split_state; size_t split_stride;   // per block: saved state of the row it started for its neighbour
+    int* split_flags;                     // per block: 1 once that state is complete (zeroed before the launch)
     EngineOpts opts;                      // the caller's per-call choice (host side only)
 };
 

@@ -357,7 +357,7 @@ obc_status hessian_tc_launch(const float* X, int d, int64_t n, int64_t ldx, floa
     return hessian_finalize_launch(partial, splits, d, H, ldh, accumulate, err, info, stream);
 }
 
-// ---- G (+)= Y X^T on the tensor cores (appendix "Sequential Quantization with OBQ": X Y^T is accumulated over
+// ---- G (+)= alpha Y X^T on the tensor cores (appendix "Sequential Quantization with OBQ": X Y^T is accumulated over
 // batches like the Hessian) ------------------------------------------------------------------------------------
 int cross_splits(int rows_a, int rows_b, int64_t n) {
     const int tiles = ((rows_a + TC_TILE - 1) / TC_TILE) * ((rows_b + TC_TILE - 1) / TC_TILE);
@@ -379,21 +379,23 @@ size_t cross_workspace_bytes(int rows_a, int rows_b, int64_t n) {
 
 __global__ void __launch_bounds__(256) cross_finalize_kernel(const float* __restrict__ partial, int splits, int rows_a,
                                                              int rows_b, float* __restrict__ G, int ldg, int accumulate,
-                                                             const int* __restrict__ err, int32_t* __restrict__ info) {
+                                                             float alpha, const int* __restrict__ err,
+                                                             int32_t* __restrict__ info) {
     const int i = blockIdx.y;
     const int j = blockIdx.x * 256 + threadIdx.x;
     if (info && i == 0 && j == 0) info[0] = (err && *err != 0) ? (int32_t)OBC_ERR_TIMEOUT : 0;
     if (j >= rows_b) return;
     float s = 0.f;
     for (int z = 0; z < splits; ++z) s += partial[(size_t)z * rows_a * rows_b + (size_t)i * rows_b + j];
+    s *= alpha;
     if (accumulate) s += G[(size_t)i * ldg + j];
     if (err && *err != 0) s = __int_as_float(0x7fc00000);
     G[(size_t)i * ldg + j] = s;
 }
 
 obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float* X, int rows_b, int64_t ldx, int64_t n,
-                           float* G, int ldg, int accumulate, obc_prec prec, int32_t* info, int wait_limit, void* ws,
-                           cudaStream_t stream) {
+                           float* G, int ldg, int accumulate, float alpha, obc_prec prec, int32_t* info, int wait_limit,
+                           void* ws, cudaStream_t stream) {
     const int wl = resolve_wait_limit(wait_limit);
     const int splits = cross_splits(rows_a, rows_b, n);
     char* p = reinterpret_cast<char*>(ws);
@@ -435,7 +437,7 @@ obc_status cross_tc_launch(const float* Y, int rows_a, int64_t ldy, const float*
     }
     OBC_CUDA_TRY(cudaGetLastError());
     dim3 fgrid((rows_b + 255) / 256, rows_a);
-    cross_finalize_kernel<<<fgrid, 256, 0, stream>>>(partial, splits, rows_a, rows_b, G, ldg, accumulate, err, info);
+    cross_finalize_kernel<<<fgrid, 256, 0, stream>>>(partial, splits, rows_a, rows_b, G, ldg, accumulate, alpha, err, info);
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;

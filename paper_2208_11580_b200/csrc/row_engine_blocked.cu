@@ -20,6 +20,14 @@
 // the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
 // finishes on chip with step-by-step updates.
 //
+// Shares of rows.  When a launch has more rows than resident blocks and the rows do not divide evenly, whole waves
+// would leave most SMs idle through the last one.  Instead every block gets the same amount of work: the rows
+// are laid end to end and cut into gridDim.x equal pieces.  A row that straddles a cut is started by the block before
+// the cut -- as that block's FIRST item -- up to a flush boundary near the cut, where its state (weights, diagonal,
+// slot map; the triangle stays in a buffer of its own) is saved, and it is finished by the next block as that
+// block's LAST item.  The state is complete long before it is needed; the reader still checks a flag with a bounded
+// wait (a cooperative launch keeps all blocks resident) and reports a row it could not pick up through row_status.
+//
 // Step protocol.  Between two flushes every slot belongs to one thread (groups of 4 consecutive slots per
 // thread), which is the only one to touch wd[j], dg[j], perm[j] and its entries of the pending vectors; the
 // update phase also leaves an FP32 estimate of each own slot's next score in registers.  Each thread proposes its best slot, the
@@ -39,6 +47,7 @@ constexpr int BLK_OFF_MV = 2048;              // int mv[64]   live slots that mo
 constexpr int BLK_OFF_CM = 2304;
 constexpr int BLK_OFF_RF = 2944;              // float rf[64]  min/max reduction of the compound grid
 constexpr int BLK_OFF_GRP = 3200;             // forced groups: int slot[4], float M[4][4] (pivot columns at the pivot slots)
+constexpr int BLK_OFF_SCHED = 3280;           // int[12]: kind of the item in work (shares of rows)
 constexpr int BLK_FIXED = 3328;
 constexpr int BLK_GS = 4;                     // forced eliminations taken together
 
@@ -53,6 +62,112 @@ __host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm =
 // flush (4 vectors x 8 consecutive slots per load) touch 32 different banks.
 __host__ __device__ inline int blk_ldz(int m) { return ((m + 8 + 31) & ~31) + 8; }     // >= m + 16
 static size_t blk_tail_bytes(int ms) { return (size_t)12 * ((ms + 3) & ~3) + (size_t)4 * ms * (ms + 1); }
+
+// ---- shares of rows ------------------------------------------------------------------------------------------------
+constexpr int BLK_SPLIT_WAIT_LIMIT = 1 << 22;  // polls (256 ns apart) before a block gives up on a row its neighbour started
+struct SplitHeader {                          // what the block that started a row leaves for the one that finishes it
+    int s_cut;                                // steps done (0: the row was not started)
+    int m0;                                   // live slots, all in [0, m0), nothing pending
+    int done;                                 // 1: nothing is left to do (the row was finished, or failed and was reported)
+    int pad[61];
+};
+// followed by: double wd[cap], double dg[cap], int perm[cap], float wfull[cap]
+__host__ __device__ inline size_t blk_split_stride(int cap) { return sizeof(SplitHeader) + (size_t)28 * cap + 256; }
+
+// Work model of a row, in units of "half a matrix element moved by a flush": a pass over the compacted triangle of m
+// slots costs m^2 / 2, a deferred-update step costs as much as BLK_STEP_COST of those (measured on B200: a pass takes
+// 1.1 - 1.3e-10 s per m^2; a step 7 us with one 512-thread row per SM, 3.4 us with several smaller blocks per SM).
+__host__ __device__ inline double blk_step_cost(int nt) { return nt >= 512 ? 30000.0 : 14000.0; }
+
+// The flush boundary of a row's schedule at which about num/den of the row's work is done (0: before the first
+// boundary; total: the share reaches into the on-chip end of the row, which is then left to the starting block).
+// Every thread of a block computes the same value from the same arguments.
+__device__ __noinline__ int blk_cut_step(int d, int ms, int total, int panel_floats, int max_pending, int g_vectors,
+                                        int num, int den, double step_cost) {
+    double all = 0.0, at = 0.0;
+    int cut = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        int m = d, s = 0;
+        double cost = 0.0;
+        while (s < total && m > ms) {
+            int b = min(max_pending, panel_floats / blk_ldz(m) + g_vectors);
+            b = max(1, min(b, min(m - ms, total - s)));
+            cost += step_cost * b;
+            s += b; m -= b;
+            if (s >= total) break;
+            cost += 0.5 * (double)m * (double)m;                  // the pass over the compacted triangle
+            if (pass == 1 && m > ms && cost <= at) cut = s;       // last boundary not beyond the share
+        }
+        cost += step_cost * 0.6 * (total - s);                    // steps on chip
+        if (pass == 0) { all = cost; at = all * (double)num / (double)den; }
+    }
+    return cut;
+}
+
+// The it-th item of block `blk` out of `ng` when `rows` rows are shared out: false when there is none.  Without
+// shares: whole rows blk, blk + ng, ...  With shares: positions in units of 1/ng of a row, row r covers
+// [r ng, (r+1) ng) and the block covers [blk rows, (blk+1) rows); the row that straddles the upper cut is started first
+// (head_num/ng of it), the one that straddles the lower cut is finished last.  Plain integer arithmetic, recomputed
+// per item so that nothing of it stays in registers during a row.
+enum { ITEM_FULL = 0, ITEM_HEAD = 1, ITEM_TAIL = 2 };
+__device__ __forceinline__ bool blk_item(bool split, int blk, int ng, int rows, int it, int* rr, int* kind, int* head_num) {
+    *kind = ITEM_FULL; *head_num = 0;
+    if (!split) { *rr = blk + it * ng; return *rr < rows; }
+    const long long a0 = (long long)blk * rows, a1 = a0 + rows;
+    const int r_first = (int)(a0 / ng), tail_num = (int)(a0 - (long long)r_first * ng);
+    const int r_last = (int)((a1 - 1) / ng);
+    int hn = (int)(a1 - (long long)r_last * ng);
+    if (hn == ng) hn = 0;                                          // the row ends at the cut: a whole row
+    const int full_lo = tail_num ? r_first + 1 : r_first, full_hi = hn ? r_last : r_last + 1;
+    const int n_items = (hn ? 1 : 0) + (full_hi - full_lo) + (tail_num ? 1 : 0);
+    if (it >= n_items) return false;
+    if (hn && it == 0) { *rr = r_last; *kind = ITEM_HEAD; *head_num = hn; }
+    else if (tail_num && it == n_items - 1) { *rr = r_first; *kind = ITEM_TAIL; }
+    else *rr = full_lo + it - (hn ? 1 : 0);
+    return true;
+}
+
+// The cold paths of the hand-over are kept out of line, so that the register allocation of a row's loop is the
+// same with and without them.
+// Thread 0: wait (bounded) for the flag of the block that started the row; returns 1 when it is set.
+__device__ __noinline__ int blk_wait_flag(int* flag) {
+    int ok = 0;
+    for (int spin = 0; spin < BLK_SPLIT_WAIT_LIMIT; ++spin) {
+        if (atomicAdd(flag, 0) != 0) { ok = 1; break; }
+        __nanosleep(256);
+    }
+    __threadfence();
+    return ok;
+}
+// Thread 0: publish the header of the row this block started (or declined to start), then the flag.
+__device__ __noinline__ void blk_publish(char* state, int* flag, int s_cut, int m0, int done) {
+    SplitHeader* sh = reinterpret_cast<SplitHeader*>(state);
+    sh->s_cut = s_cut; sh->m0 = m0; sh->done = done;
+    __threadfence();
+    atomicExch(flag, 1);
+}
+// All threads: state of a row between shared memory and the hand-over record (save = true: to the record).
+__device__ __noinline__ void blk_state_copy(bool save, char* state, int cap, int d, int m, int nt, double* wd, double* dg,
+                                            int* perm, unsigned short* srcm, float* wfull) {
+    char* base = state + sizeof(SplitHeader);
+    double* swd = reinterpret_cast<double*>(base);
+    double* sdg = swd + cap;
+    int* sperm = reinterpret_cast<int*>(sdg + cap);
+    float* swf = reinterpret_cast<float*>(sperm + cap);
+    const int tid = threadIdx.x;
+    if (save) {
+        for (int j = tid; j < m; j += nt) { swd[j] = wd[j]; sdg[j] = dg[j]; sperm[j] = perm[j]; }
+        if (wfull) for (int j = tid; j < d; j += nt) swf[j] = wfull[j];
+        __threadfence();                   // state, triangle and outputs of every thread before the flag
+    } else {
+        for (int j = tid; j < cap; j += nt) {
+            const bool in = j < m;
+            wd[j] = in ? swd[j] : 0.0; dg[j] = in ? sdg[j] : 0.0; perm[j] = in ? sperm[j] : -1;
+            srcm[j] = (unsigned short)j;
+            if (wfull && j < d) wfull[j] = swf[j];
+        }
+    }
+}
 
 struct Records {                              // views into one record buffer
     unsigned* key; int* slot; int* orig; double* s; double* w; double* dgv;
@@ -363,9 +478,9 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 __device__ __forceinline__ uint32_t tf32_rn(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 __device__ __forceinline__ void tf32_split(float x, uint32_t& hi, uint32_t& lo) {
     hi = tf32_rn(x);                                        // 11 significant bits
-    // the difference is exact in FP32 and has either sign; the tensor core reads its leading 11 bits (truncation of
-    // a part whose sign is random is no bias)
-    lo = __float_as_uint(x - __uint_as_float(hi));
+    // the difference is exact in FP32 (up to 13 significant bits, either sign); it is rounded to nearest as well, so
+    // that hi + lo represents x to 2^-24 instead of the 2^-23 the tensor core's truncation of its input would leave
+    lo = tf32_rn(x - __uint_as_float(hi));
 }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -447,10 +562,15 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                 for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
 #pragma unroll
                 for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bh[n][0], bh[n][1]);
+                // That one truncation per partial sum still shortens every increment by half a unit in the last place on
+                // average, the same way for every element and pass -- a uniform scaling of all Lemma-1 updates, which the
+                // last steps of a row (the few remaining entries carry everything eliminated before) amplify: measured
+                // on a 2304-column layer, the final loss was off by 1.7e-4 with it and 1.3e-5 without.  Setting the last
+                // mantissa bit turns "truncated" into "truncated + 0 or 1 unit", which is right on average.
 #pragma unroll
                 for (int n = 0; n < 8; ++n)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[n][e] += dk[n][e];
+                    for (int e = 0; e < 4; ++e) acc[n][e] += __uint_as_float(__float_as_uint(dk[n][e]) | 1u);
             }
             // ---- the tile of H (in L2 by now: the cursor passed it two tiles ago), minus the increment -----------
             float4 hv[4][2];
@@ -556,7 +676,9 @@ __device__ __forceinline__ double block4_score(const double* w, const double* a,
 // barriers per four steps, each pending vector read once for four columns.  Same arithmetic per element as four
 // single steps except that a column's corrections are subtracted one by one instead of summed first.
 // GPV = the kernel can keep further pending vectors in global memory (very long rows, 512 threads only).
-template <int NT, int KMAX, bool Q, int BC, bool FG, bool GPV>
+// SH = the kernel takes shares of rows (a row may be started by one block and finished by the next); launches whose
+// rows divide evenly over the blocks run the kernel built without that code.
+template <int NT, int KMAX, bool Q, int BC, bool FG, bool GPV, bool SH>
 __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const EngineArgs a) {
     extern __shared__ __align__(16) char smem[];
     constexpr int NW = NT / 32;
@@ -588,17 +710,33 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     float* tlr = tu + msr;
     float* S = tlr + msr;
     const int lds = ms + 1;
-    float* Hp = a.Hws ? a.Hws + (size_t)blockIdx.x * d * a.ldp : nullptr;
     const int ldp = a.ldp;
+    float* const Hp0 = a.Hws ? a.Hws + (size_t)blockIdx.x * d * a.ldp : nullptr;      // the block's own triangle
+#define HP (SH ? (a.Hws + (size_t)reinterpret_cast<const int*>(smem + BLK_OFF_SCHED)[2] * d * ldp) : Hp0)
     // overflow of the pending vectors: gB more of them in global memory (sized to stay in L2), stride gld
     // (only the one-row-per-SM configuration uses it; the other kernels are built without that code)
     constexpr bool GP = GPV;
     const int gB = (GP && a.Gpan) ? a.g_vectors : 0, gld = a.g_ld;
-    float* G = (GP && a.Gpan) ? a.Gpan + (size_t)blockIdx.x * a.g_vectors * a.g_ld : nullptr;
-    float* zstage = panel + a.panel_floats + (size_t)warp * a.g_vectors * 16;    // per warp: g_vectors x 16 floats
+    // (recomputed at every use instead of held in registers: the kernels with the overflow code have none to spare)
+#define GVEC (a.Gpan + (size_t)blockIdx.x * a.g_vectors * a.g_ld)
+#define ZSTAGE (panel + a.panel_floats + (size_t)warp * a.g_vectors * 16)      /* per warp: g_vectors x 16 floats */
 
-    for (int rr = blockIdx.x; rr < a.row_count; rr += gridDim.x) {
+    // ---- this block's items: whole rows, plus (shares of rows) the start of one row and the rest of another -------
+    int* sched = reinterpret_cast<int*>(smem + BLK_OFF_SCHED);
+    if (SH) {                                  // the item counter lives in shared memory too
+        if (tid == 0) sched[3] = 0;
+        __syncthreads();
+    }
+    for (int it_reg = 0;; ++it_reg) {
+        int rr, kind, head_num;
+        const int it = SH ? sched[3] : it_reg;
+        if (SH) { __syncthreads(); if (tid == 0) sched[3] = it + 1; __syncthreads(); }    // read by all, then moved on
+        if (!blk_item(SH, blockIdx.x, gridDim.x, a.row_count, it, &rr, &kind, &head_num)) break;
+        const int NG = gridDim.x;
         const int r = a.row_begin + rr;
+        // the triangle of the row in work: buffer blk for whole rows, ng + blk for the row this block starts, ng + blk - 1
+        // for the row it finishes (kept in shared memory and re-read where needed, not in registers)
+        int hbuf = kind == ITEM_FULL ? (int)blockIdx.x : (kind == ITEM_HEAD ? NG + (int)blockIdx.x : NG + (int)blockIdx.x - 1);
         int n_forced = 0, n_free = 0;
         bool quant = false;
         if (a.mode == MODE_PRUNE) { n_free = a.steps; }
@@ -611,7 +749,49 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         const int total = n_forced + n_free;
         const bool outliers = Q && quant && (a.flags & OBC_FLAG_OUTLIERS);
 
+        // ---- shares of rows: where this item stops, and what a continued row starts from -----------------
+        int s_stop = total;                // steps [s_begin, s_stop) of the row are this item's
+        int s_begin = 0, m_begin = d;
+        if (kind == ITEM_HEAD) s_stop = blk_cut_step(d, ms, total, a.panel_floats, a.max_pending, gB, head_num, NG, blk_step_cost(NT));
+        if (kind == ITEM_HEAD && s_stop <= 0) {
+            // too small a share to be worth a start: the neighbour takes the whole row
+            if (tid == 0) blk_publish(a.split_state + (size_t)blockIdx.x * a.split_stride, a.split_flags + blockIdx.x, 0, d, 0);
+            continue;
+        }
+        if (kind == ITEM_TAIL) {
+            const SplitHeader* sh = reinterpret_cast<const SplitHeader*>(a.split_state + (size_t)(blockIdx.x - 1) * a.split_stride);
+            if (tid == 0) bc->nh = blk_wait_flag(a.split_flags + blockIdx.x - 1);
+            __syncthreads();
+            const int ok = bc->nh;
+            __syncthreads();
+            if (!ok) {                     // the start of this row never arrived: report it, touch nothing else
+                if (tid == 0) a.row_status[r] = -(int)OBC_ERR_TIMEOUT;
+                continue;
+            }
+            if (sh->done) continue;        // finished (or failed and reported) by the block that started it
+            s_begin = sh->s_cut; m_begin = sh->m0;
+            if (s_begin == 0) { kind = ITEM_FULL; hbuf = (int)blockIdx.x; }    // never started: a whole row
+        }
+
+        if (SH) {                              // read during and after the row
+            if (tid == 0) { sched[0] = kind; sched[1] = s_stop; sched[2] = hbuf; }
+            __syncthreads();
+        }
+
         // ---- row set-up ------------------------------------------------------------------------------
+        if (kind == ITEM_TAIL) {
+            // continue a row: state as saved at the flush boundary s_begin (slots [0, m_begin) all live, nothing pending)
+            blk_state_copy(false, a.split_state + (size_t)(blockIdx.x - 1) * a.split_stride, cap, d, m_begin, NT, wd, dg, perm, srcm,
+                           has_wfull ? wfull : nullptr);
+            for (int k = tid; k < 160; k += NT) colmask[k] = 0u;
+            if (tid == 0) {
+                bc->sc = 1.0; bc->ze = 0.0; bc->mq = 0.0;
+                if (a.mode == MODE_QUANT || (a.mode == MODE_REPLAY_QUANT && s_begin > n_forced)) {
+                    bc->sc = (double)a.scale[r]; bc->ze = (double)a.zero[r];
+                    bc->mq = (double)grid_maxq(a.bits, a.symmetric);
+                }
+            }
+        } else {
         for (int j = tid; j < d; j += NT) {
             const float w = a.W[(size_t)r * a.ldw + j];
             wd[j] = (double)w;
@@ -643,11 +823,12 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         if (a.w_trace)
             for (int j = tid; j < d; j += NT)
                 a.w_trace[((size_t)r * (a.trace_steps + 1)) * d + j] = a.W[(size_t)r * a.ldw + j];
+        }
         bool tail = false;
-        if (d > ms && total > 0) {
+        if (kind != ITEM_TAIL && d > ms && total > 0) {
             for (int i = warp; i < d; i += NW) {
                 const float4* s4 = reinterpret_cast<const float4*>(a.Hinv + (size_t)i * a.ldhi);
-                float4* d4 = reinterpret_cast<float4*>(Hp + (size_t)i * ldp);
+                float4* d4 = reinterpret_cast<float4*>(HP + (size_t)i * ldp);
                 const int n4 = (i >> 2) + 1;
                 if (GP || (FG && NT >= 512)) {      // (kernels with no registers to spare: one load in flight)
                     for (int j4 = lane; j4 < n4; j4 += 32) d4[j4] = s4[j4];
@@ -665,13 +846,13 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         __syncthreads();
         double gsc = bc->sc, gze = bc->ze, gmq = bc->mq;       // grid parameters of the row (registers)
 
-        int m0 = d;                      // slots in use (tail phase: number of live slots)
+        int m0 = m_begin;                // slots in use (tail phase: number of live slots)
         int nb = 0;                      // pending vectors
         int ldz = blk_ldz(m0);
         int scap = a.panel_floats / ldz;     // pending vectors that fit into shared memory at this row length
         int bcur = min(a.max_pending, scap + gB);
         if (BC) bcur &= ~(BC - 1);           // whole blocks between two flushes, so that 4-slot groups stay together
-        int s = 0;
+        int s = s_begin;
         bool failed = false;
         int blk_base = 0;                // block pruning: first slot and score of the block being eliminated
         double blk_score = 0.0;
@@ -683,7 +864,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         double gisc = 1.0 / gsc;
         for (; s < total; ++s) {
             if (!tail) {
-                if (d > ms && nb > 0 && (nb == bcur || m0 - nb <= ms)) {
+                if (d > ms && nb > 0 && (nb == bcur || m0 - nb <= ms || (SH && s == sched[1]))) {
                     // ---- flush: apply the pending vectors and compact to m1 slots ------------------------
                     __syncthreads();                           // the last step's vector and perm updates
                     const int m1 = m0 - nb;
@@ -702,7 +883,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     const int nh = bc->nh;
                     for (int idx = tid; idx < nh * nb; idx += NT) {
                         const int q = idx / nb, b = idx - q * nb;
-                        float* zr = (!GP || b < scap) ? panel + (size_t)b * ldz : G + (size_t)(b - scap) * gld;
+                        float* zr = (!GP || b < scap) ? panel + (size_t)b * ldz : GVEC + (size_t)(b - scap) * gld;
                         zr[hl[q]] = zr[mv[q]];
                     }
                     if (tid < nh) {
@@ -712,9 +893,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     }
                     __syncthreads();
                     if (!GP || nb <= scap)
-                        blk_flush_mma<NT, true>(Hp, ldp, m1, nb, panel, ldz, srcm, colmask);      // evict-first at every row length (~1 %)
+                        blk_flush_mma<NT, true>(HP, ldp, m1, nb, panel, ldz, srcm, colmask);      // evict-first at every row length (~1 %)
                     else
-                        blk_flush<NT, 16, (NT >= 512)>(Hp, ldp, m1, nb, min(nb, scap), panel, ldz, G, gld, zstage, srcm, colmask);
+                        blk_flush<NT, 16, (NT >= 512)>(HP, ldp, m1, nb, min(nb, scap), panel, ldz, GVEC, gld, ZSTAGE, srcm, colmask);
                     __syncthreads();
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
@@ -736,9 +917,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     if (BC) bcur &= ~(BC - 1);
                     __syncthreads();
                 }
+                if (SH && s == sched[1]) break;      // (shares of rows) the row is handed over here, everything applied
                 if (m0 <= ms) {
                     // ---- move on chip: slots [0, m0) are all live here and the stored triangle is current
-                    const float* src = (d > ms) ? Hp : a.Hinv;
+                    const float* src = (d > ms) ? HP : a.Hinv;
                     const int sld = (d > ms) ? ldp : a.ldhi;
                     for (int i = warp; i < m0; i += NW)
                         for (int j = lane; j <= i; j += 32) S[i * lds + j] = src[(size_t)i * sld + j];
@@ -748,7 +930,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             }
             const bool forced = s < n_forced;
             const bool q_now = Q && quant && !forced;
-            if (FG && forced && !tail && !has_wfull && !has_nm && s + BLK_GS <= n_forced && nb + BLK_GS <= bcur &&
+            if (FG && forced && !tail && !has_wfull && !has_nm && s + BLK_GS <= (SH ? min(n_forced, sched[1]) : n_forced) && nb + BLK_GS <= bcur &&
                 (!GP || nb + BLK_GS <= scap)) {
                 // ======================= four forced eliminations together ================================
                 constexpr int GS = BLK_GS;
@@ -800,7 +982,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 #pragma unroll
                         for (int g = 0; g < GS; ++g) {
                             const int p = p4[g];
-                            const float* rowp = Hp + (size_t)p * ldp;
+                            const float* rowp = HP + (size_t)p * ldp;
                             if (jb + 3 <= p) {
                                 const float4 t = *reinterpret_cast<const float4*>(rowp + jb);
                                 v[g][4 * g4] = t.x; v[g][4 * g4 + 1] = t.y; v[g][4 * g4 + 2] = t.z; v[g][4 * g4 + 3] = t.w;
@@ -808,7 +990,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 #pragma unroll
                                 for (int q = 0; q < 4; ++q) {
                                     const int j = jb + q;
-                                    if ((live >> (4 * g4 + q)) & 1u) v[g][4 * g4 + q] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                                    if ((live >> (4 * g4 + q)) & 1u) v[g][4 * g4 + q] = (j <= p) ? rowp[j] : HP[(size_t)j * ldp + p];
                                 }
                             }
                         }
@@ -849,7 +1031,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     // the four eliminations at the pivot slots themselves (every thread, same values)
                     float zz[GS][GS];                      // vector e at pivot slot x
                     double idp[GS], fg[GS];
-                    float rsq[GS];
+                    double rsq[GS];
                     bool fine = true;
 #pragma unroll
                     for (int g = 0; g < GS; ++g) {
@@ -864,9 +1046,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         if (!(dpp > 0.0) || !isfinite(dpp) || !isfinite(w)) fine = false;
                         idp[g] = 1.0 / dpp;
                         fg[g] = w * idp[g];
-                        rsq[g] = __frsqrt_rn((float)dpp);
+                        const double r0 = (double)__frsqrt_rn((float)dpp);
+                        rsq[g] = r0 * (1.5 - 0.5 * dpp * r0 * r0);
 #pragma unroll
-                        for (int x = 0; x < GS; ++x) zz[g][x] = mc[x] * rsq[g];
+                        for (int x = 0; x < GS; ++x) zz[g][x] = __double2float_rn((double)mc[x] * rsq[g]);
 #pragma unroll
                         for (int x = g + 1; x < GS; ++x) {
                             wp4[x] -= fg[g] * (double)mc[x];
@@ -897,7 +1080,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                                         for (int e = 0; e < g; ++e) vj = fmaf(-zv[e][q], zz[e][g], vj);
                                         nw -= fg[g] * (double)vj;
                                         nd -= (double)vj * (double)vj * idp[g];
-                                        zv[g][q] = vj * rsq[g];
+                                        zv[g][q] = __double2float_rn((double)vj * rsq[g]);
                                     }
                                 }
                                 if (gm < GS) perm[j] = -1;
@@ -996,11 +1179,11 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             const double e = wp - qp;
             if (!tail) {
                 // ======================= deferred-update step ==============================================
-                float* zb = (!GP || nb < scap) ? panel + (size_t)nb * ldz : G + (size_t)(nb - scap) * gld;
+                float* zb = (!GP || nb < scap) ? panel + (size_t)nb * ldz : GVEC + (size_t)(nb - scap) * gld;
                 // pivot column of the stored matrix (own slots), corrected by the pending vectors
                 float c[KMAX], corr[KMAX];
                 unsigned live = 0u;
-                const float* rowp = Hp + (size_t)p * ldp;
+                const float* rowp = HP + (size_t)p * ldp;
 #pragma unroll
                 for (int g = 0; g < KMAX / 4; ++g) {
                     const int jb = own_slot<NT>(4 * g);
@@ -1019,13 +1202,16 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const int j = jb + q;
-                            if ((live >> (4 * g + q)) & 1u) c[4 * g + q] = (j <= p) ? rowp[j] : Hp[(size_t)j * ldp + p];
+                            if ((live >> (4 * g + q)) & 1u) c[4 * g + q] = (j <= p) ? rowp[j] : HP[(size_t)j * ldp + p];
                         }
                     }
                 }
                 const double idpp = 1.0 / dpp;
                 const double f = e * idpp;
-                const float rs = __frsqrt_rn((float)dpp);
+                // 1/sqrt(dpp) to FP64 accuracy (one Newton step on the FP32 estimate): the pending vector z = v / sqrt(dpp)
+                // is then rounded once per entry, with no error common to the whole rank-1 term z z^T
+                const double rs0 = (double)__frsqrt_rn((float)dpp);
+                const double rs = rs0 * (1.5 - 0.5 * dpp * rs0 * rs0);
                 const int nbs = GP ? min(nb, scap) : nb;
                 for (int b = 0; b < nbs; ++b) {
                     const float* zo = panel + (size_t)b * ldz;
@@ -1044,7 +1230,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 if (GP)
 #pragma unroll 2
                 for (int b = nbs; b < nb; ++b) {               // the overflow vectors, from L2
-                    const float* zo = G + (size_t)(b - scap) * gld;
+                    const float* zo = GVEC + (size_t)(b - scap) * gld;
                     const float zp = zo[p];
 #pragma unroll
                     for (int g = 0; g < KMAX / 4; ++g) {
@@ -1083,7 +1269,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         const double nw = wd[j] - f * (double)vj;
                         const double nd = dg[j] - (double)vj * (double)vj * idpp;
                         wd[j] = nw; dg[j] = nd;
-                        zv[q] = vj * rs;
+                        zv[q] = __double2float_rn((double)vj * rs);
                         if (est_next) sa[k] = score_estimate<Q>(nw, nd, q_next, gsc, gisc, gze, gmq);
                         if (has_nm) {
                             if ((pq[q] >> nm_lg) == (op >> nm_lg)) cntw[g] += 1u << (8 * q);
@@ -1169,6 +1355,19 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
         }
         // ---- row epilogue ---------------------------------------------------------------------------------
         __syncthreads();
+        if (SH && sched[0] == ITEM_HEAD) {
+            // (shares of rows) leave the row to the next block: state at the flush boundary, then the flag
+            const bool handed = !failed && s < total;
+            if (handed)
+                blk_state_copy(true, a.split_state + (size_t)blockIdx.x * a.split_stride, cap, d, m0, NT, wd, dg, perm, srcm,
+                               has_wfull ? wfull : nullptr);
+            else
+                __threadfence();
+            __syncthreads();
+            if (tid == 0)
+                blk_publish(a.split_state + (size_t)blockIdx.x * a.split_stride, a.split_flags + blockIdx.x, s, m0, handed ? 0 : 1);
+            if (handed) { __syncthreads(); continue; }
+        }
         if (failed) {           // stopped early: report the step, mark what was not produced
             if (tid == 0) a.row_status[r] = 1 + s;
             const int t0 = (s < n_forced) ? 0 : s - n_forced;
@@ -1184,6 +1383,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     }
 }
 
+#undef HP
+#undef GVEC
+#undef ZSTAGE
 // ---- host side ---------------------------------------------------------------------------------------------
 struct BlkPlan {
     int nt;            // threads per block
@@ -1260,6 +1462,13 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     return true;
 }
 
+// The largest grid any thread-count choice uses at this row length (threads per row are bounded below by the row
+// length, see blk_plan).
+static int blk_max_blocks(int d, const DeviceInfo& di) {
+    const int cap = (d + 3) & ~3;
+    return di.sm_count * (cap > 2048 ? 1 : (cap > 1024 ? 2 : 4));
+}
+
 size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di) {
     // valid for every per-call choice: a row needs its private triangle whenever d exceeds the on-chip threshold,
     // and that threshold depends on the threads per row and on the per-row state the call keeps
@@ -1273,11 +1482,15 @@ size_t blocked_engine_workspace_bytes(int row_count, int d, const DeviceInfo& di
         }
     if (!off_chip) return 256;
     const int cap = (d + 3) & ~3;
-    int blocks = di.sm_count * 4;                 // the largest grid any thread-count choice uses
+    int blocks = blk_max_blocks(d, di);
+    // more rows than blocks: every block may also hold the row it starts for its neighbour (a second triangle),
+    // plus the saved state and the flags of the hand-over
+    const bool may_split = row_count == 0 || row_count > di.sm_count;
     if (row_count > 0 && row_count < blocks) blocks = row_count;
     const int gblocks = blocks < di.sm_count ? blocks : di.sm_count;     // overflow vectors: one block per SM only
-    return round_up((size_t)blocks * d * cap * sizeof(float), 256) +
-           round_up((size_t)gblocks * BLK_MAXB * ((cap + 15) & ~15) * sizeof(float), 256);
+    return round_up((size_t)blocks * (may_split ? 2 : 1) * d * cap * sizeof(float), 256) +
+           round_up((size_t)gblocks * BLK_MAXB * ((cap + 15) & ~15) * sizeof(float), 256) +
+           (may_split ? round_up((size_t)blocks * blk_split_stride(cap), 256) + round_up((size_t)blocks * sizeof(int), 256) : 0);
 }
 
 obc_status blocked_engine_plan(int d, int with_trace, int row_count, const EngineOpts& eo, int32_t* plan) {
@@ -1293,33 +1506,51 @@ obc_status blocked_engine_plan(int d, int with_trace, int row_count, const Engin
 }
 
 template <int NT, int KMAX, bool Q, int BC, bool FG, bool GPV>
-static obc_status blk_launch_g(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    OBC_CUDA_TRY(cudaFuncSetAttribute(blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV>,
-                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV><<<blocks, NT, smem, stream>>>(a);
+static obc_status blk_launch_g(EngineArgs a, int blocks, size_t smem, int sm_count, cudaStream_t stream) {
+    auto kernel = blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV, false>;
+    auto kernel_sh = blocked_engine_kernel<NT, KMAX, Q, BC, FG, GPV, (BC == 0)>;     // (block pruning takes no shares)
+    if (a.split) {
+        // A block may wait (bounded) for the row its neighbour started, so all blocks must be resident at once: checked
+        // here, and guaranteed by a cooperative launch.  If the grid does not fit, rows run in whole waves instead.
+        OBC_CUDA_TRY(cudaFuncSetAttribute(kernel_sh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int per_sm = 0;
+        OBC_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel_sh, NT, smem));
+        int coop = 0, dev = 0;
+        OBC_CUDA_TRY(cudaGetDevice(&dev));
+        OBC_CUDA_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+        if (BC != 0 || !coop || (long long)per_sm * sm_count < blocks) a.split = 0;
+    }
+    if (a.split) {
+        OBC_CUDA_TRY(cudaMemsetAsync(a.split_flags, 0, (size_t)blocks * sizeof(int), stream));
+        void* params[1] = {(void*)&a};
+        OBC_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kernel_sh, dim3(blocks), dim3(NT), params, smem, stream));
+    } else {
+        OBC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kernel<<<blocks, NT, smem, stream>>>(a);
+    }
     count_launch();
     OBC_CUDA_TRY(cudaGetLastError());
     return OBC_OK;
 }
 
 template <int NT, int KMAX, bool Q, int BC, bool FG>
-static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    if (NT >= 512 && a.Gpan != nullptr) return blk_launch_g<NT, KMAX, Q, BC, FG, (NT >= 512)>(a, blocks, smem, stream);
-    return blk_launch_g<NT, KMAX, Q, BC, FG, false>(a, blocks, smem, stream);
+static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, int sm_count, cudaStream_t stream) {
+    if (NT >= 512 && a.Gpan != nullptr) return blk_launch_g<NT, KMAX, Q, BC, FG, (NT >= 512)>(a, blocks, smem, sm_count, stream);
+    return blk_launch_g<NT, KMAX, Q, BC, FG, false>(a, blocks, smem, sm_count, stream);
 }
 
 template <int NT, int KMAX>
-static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, cudaStream_t stream) {
-    if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4, false>(a, blocks, smem, stream);
+static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, int sm_count, cudaStream_t stream) {
+    if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4, false>(a, blocks, smem, sm_count, stream);
     switch (a.mode) {                       // the replay modes are the ones with forced eliminations
-        case MODE_QUANT:        return blk_launch_q<NT, KMAX, true, 0, false>(a, blocks, smem, stream);
+        case MODE_QUANT:        return blk_launch_q<NT, KMAX, true, 0, false>(a, blocks, smem, sm_count, stream);
         // (with 512 threads the OBQ kernel has no registers to spare for the four columns: single steps there)
-        case MODE_REPLAY_QUANT: return blk_launch_q<NT, KMAX, true, 0, (NT <= 256)>(a, blocks, smem, stream);
-        case MODE_REPLAY:       return blk_launch_q<NT, KMAX, false, 0, true>(a, blocks, smem, stream);
-        default:                return blk_launch_q<NT, KMAX, false, 0, false>(a, blocks, smem, stream);
+        case MODE_REPLAY_QUANT: return blk_launch_q<NT, KMAX, true, 0, (NT <= 256)>(a, blocks, smem, sm_count, stream);
+        case MODE_REPLAY:       return blk_launch_q<NT, KMAX, false, 0, true>(a, blocks, smem, sm_count, stream);
+        default:                return blk_launch_q<NT, KMAX, false, 0, false>(a, blocks, smem, sm_count, stream);
     }
 }
-static obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream);
+static obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, int sm_count, cudaStream_t stream);
 
 obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaStream_t stream) {
     DeviceInfo di;
@@ -1347,23 +1578,37 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     a.g_vectors = 0;
     a.g_ld = p.g_ld;
     a.ldp = a.cap;
+    a.split = 0;
+    a.split_state = nullptr; a.split_flags = nullptr; a.split_stride = 0;
     if (a.d > a.ms) {
-        const size_t tri = round_up((size_t)blocks * a.d * a.cap * sizeof(float), 256);
+        // Shares of rows (equal work per block instead of whole waves): when there are more rows than blocks and they
+        // do not divide evenly; not with the N:M pattern or block pruning, whose extra per-row state is not handed over.
+        const bool want_split = a.row_count > blocks && a.row_count % blocks != 0 && a.nm_prune == 0 && !bc &&
+                                !(a.opts.flags & OBC_ENGINE_WHOLE_WAVES);
+        const size_t tri = round_up((size_t)blocks * (want_split ? 2 : 1) * a.d * a.cap * sizeof(float), 256);
         const size_t gpan = p.g_vectors ? round_up((size_t)blocks * p.g_vectors * p.g_ld * sizeof(float), 256) : 0;
-        if (!ws || !aligned256(ws) || ws_bytes < tri + gpan) return OBC_ERR_WORKSPACE;
+        const size_t sst = want_split ? round_up((size_t)blocks * blk_split_stride(a.cap), 256) : 0;
+        const size_t sfl = want_split ? round_up((size_t)blocks * sizeof(int), 256) : 0;
+        if (!ws || !aligned256(ws) || ws_bytes < tri + gpan + sst + sfl) return OBC_ERR_WORKSPACE;
         a.Hws = reinterpret_cast<float*>(ws);
         if (p.g_vectors) {
             a.Gpan = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + tri);
             a.g_vectors = p.g_vectors;
         }
+        if (want_split) {
+            a.split = 1;
+            a.split_state = reinterpret_cast<char*>(ws) + tri + gpan;
+            a.split_stride = blk_split_stride(a.cap);
+            a.split_flags = reinterpret_cast<int*>(reinterpret_cast<char*>(ws) + tri + gpan + sst);
+        }
     }
-    return blk_launch_nt(a, p.nt, blocks, p.smem, stream);
+    return blk_launch_nt(a, p.nt, blocks, p.smem, di.sm_count, stream);
 }
 
-obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, cudaStream_t stream) {
-    if (nt == 128) return blk_launch<128, 8>(a, blocks, smem, stream);
-    if (nt == 256) return blk_launch<256, 8>(a, blocks, smem, stream);
-    return blk_launch<512, 12>(a, blocks, smem, stream);
+obc_status blk_launch_nt(const EngineArgs& a, int nt, int blocks, size_t smem, int sm_count, cudaStream_t stream) {
+    if (nt == 128) return blk_launch<128, 8>(a, blocks, smem, sm_count, stream);
+    if (nt == 256) return blk_launch<256, 8>(a, blocks, smem, sm_count, stream);
+    return blk_launch<512, 12>(a, blocks, smem, sm_count, stream);
 }
 
 }  // namespace obc

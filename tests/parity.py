@@ -14,6 +14,7 @@ import numpy as np
 import oracle
 
 MARGIN_TOL = 1e-6      # picks must agree wherever best and forced scores differ by more than this (relative)
+OBQ_GATE_CAP = 4e-5    # upper limit of the OBQ pick gate (see check_rows)
 REL_TOL = 1e-4         # loss traces and weights: relative error bound in FP32.  Weights are compared relative to
                        # max(|reference entry|, largest initial weight of the row): late in a row the few remaining
                        # weights carry the compensation of all the others and grow to several times the initial scale
@@ -46,8 +47,10 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
         # |dw| <= 2.5e-7 max|w| (4 * 2^-24), and a half-step score moves by the relative amount 4 |dw| / Delta
         # under such a perturbation.  The 1e-6 margin is therefore taken on the weight scale: picks whose
         # scores differ by less than 1e-6 * max|w| / Delta of the half-step score are ties.
+        # That bound is 1.3e-4 on an 8-bit grid; the largest gap seen at a differing pick is 1.9e-5 (the 8-bit compound
+        # configuration, streaming engine), so the gate is capped at about twice that.
         wmax = np.abs(W).max(axis=1, keepdims=True)
-        tol = MARGIN_TOL * np.maximum(1.0, wmax / (2.0 * half))
+        tol = np.minimum(MARGIN_TOL * np.maximum(1.0, wmax / (2.0 * half)), OBQ_GATE_CAP)
     else:
         tol = MARGIN_TOL
     bad = differ & (gap > tol)
@@ -129,10 +132,10 @@ class WithEngineOpts:
     _ENGINE_CALLS = ("obc_prune_trace", "obc_prune_apply", "obc_quantize", "obc_prune_nm", "obc_prune_blocks",
                      "obc_engine_plan")
 
-    def __init__(self, module, engine=0, threads=0, max_pending=0):
+    def __init__(self, module, engine=0, threads=0, max_pending=0, flags=0):
         self._m = module
         self.engine_name = {0: "auto", 1: "streaming", 2: "blocked"}.get(int(engine), str(engine))
-        self.opts = module.engine_opts(engine, threads, max_pending)
+        self.opts = module.engine_opts(engine, threads, max_pending, flags)
 
     def __getattr__(self, name):
         f = getattr(self._m, name)

@@ -79,7 +79,7 @@ def test_engine_options_are_validated_per_call(lib):
     assert trace(binding.EngineOpts(7, 0, 0, 0)) == 1          # unknown engine
     assert trace(binding.EngineOpts(2, 100, 0, 0)) == 1        # threads not 128/256/512
     assert trace(binding.EngineOpts(2, 0, 65, 0)) == 1         # more deferred updates than the kernels hold
-    assert trace(binding.EngineOpts(2, 0, 0, 1)) == 1          # reserved field
+    assert trace(binding.EngineOpts(2, 0, 0, 2)) == 1          # unknown flag
     plan = (ctypes.c_int32 * 8)()
     assert lib.obc_engine_plan(8, 0, 0, binding._opts(binding.EngineOpts(9, 0, 0, 0)), plan) == 1
     assert "obc_set_engine" not in binding.EXPORTED_SYMBOLS

@@ -554,8 +554,16 @@ def test_dense_refit_against_oracle(obc, R, d, n, prec):
     assert np.abs(G.cpu().numpy() - ref).max() <= tol * scale
     H, Hinv = gpu_hinv(obc, X, prec=prec)
     Wn = torch.zeros(R, d, dtype=torch.float32, device="cuda")
-    obc.obc_refit(G, Hinv, Wn)
+    obc.obc_refit(G, Hinv, Wn, prec=prec)                  # the product G Hinv in the same precision as the Gram matrices
     torch.cuda.synchronize()
     want = oracle.refit(X, Y, DAMP)
     wtol = {0: 2e-4, 1: 2e-2, 2: 5e-4}[prec]
     assert np.abs(Wn.cpu().numpy() - want).max() <= wtol * np.abs(want).max()
+    # the product alone, against FP64 on the same FP32 operands
+    Wf = torch.zeros(R, d, dtype=torch.float32, device="cuda")
+    obc.obc_refit(G, Hinv, Wf, prec=prec)
+    prod = 2.0 * G.cpu().numpy().astype(np.float64) @ Hinv.cpu().numpy().astype(np.float64)
+    ptol = {0: 2e-6, 1: 1e-3, 2: 2e-5}[prec]
+    pscale = 2.0 * np.sqrt((G.cpu().numpy().astype(np.float64) ** 2).sum(axis=1).max() *
+                           (Hinv.cpu().numpy().astype(np.float64) ** 2).sum(axis=1).max())
+    assert np.abs(Wf.cpu().numpy() - prod).max() <= ptol * pscale
