@@ -219,8 +219,11 @@ obc_status obc_select_global_mask(const float *loss, const int32_t *order, int d
  * (about 16.2 MiB) until the process exits.
  *   Limits: d_row <= OBC_SELECT_STATIC_MAX_ROWS and d_row*d_col <= OBC_SELECT_STATIC_MAX_KEYS; anything larger
  *   returns OBC_ERR_STATIC_SCRATCH and launches nothing.
- *   The first call on each device looks up the array's device address (a host-side runtime call, no allocation);
- *   make that first call outside any stream capture.  No call allocates or frees memory.
+ *   The first call on each device looks up the array's device address (a host-side runtime call).  With CUDA's
+ *   lazy module loading that first call may also be the moment the driver loads this library's device image and
+ *   sets the array aside, which can fail once a host application owns all remaining memory: make the first call at
+ *   start-up, before the memory is handed out and outside any stream capture (or run with CUDA_MODULE_LOADING=EAGER,
+ *   which ties the reservation to library load).  After it, no call allocates or frees memory.
  *   All calls on a device share the one array: the call rewrites everything it later reads, so back-to-back calls
  *   on one stream are fine, but two calls that can overlap on the GPU (different streams or threads) race.
  * Results are identical to obc_select_global_mask. */

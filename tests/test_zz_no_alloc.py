@@ -32,11 +32,15 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
         want_c = torch.full((R,), -1, dtype=torch.int32, device="cuda")
         want_m = torch.full((R, d), 7, dtype=torch.uint8, device="cuda")
         obc.obc_select_global_mask(L, P, k, want_c, want_m)
-        for _ in range(2):
+        for rep in range(2):
             got_c = torch.full((R,), -2, dtype=torch.int32, device="cuda")
             got_m = torch.full((R, d), 9, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             obc.obc_select_global_mask_static(L, P, k, got_c, got_m)
             torch.cuda.synchronize()
+            if rep == 1:      # (the very first call on a device may load the device image; later calls take nothing)
+                assert torch.cuda.mem_get_info()[0] == free_before
             assert torch.equal(got_c, want_c) and torch.equal(got_m, want_m)
         assert int(want_c.sum()) == k
 
