@@ -757,7 +757,7 @@ def main():
                          "(default: C3 when the workload is C5 on one GPU, else none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--hessian-prec", default="bf16x3", choices=["fp32", "tf32", "bf16x3"])
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-seconds", type=float, default=18.0)
     ap.add_argument("--engine", default="blocked", choices=["blocked", "streaming"],
                     help="row elimination engine: deferred block updates (default) or one pass per step")
     ap.add_argument("--threads", type=int, default=0, help="--small-case: threads per row of the blocked engine (0 = from d_col)")

@@ -478,9 +478,9 @@ __device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m
 __device__ __forceinline__ uint32_t tf32_rn(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 __device__ __forceinline__ void tf32_split(float x, uint32_t& hi, uint32_t& lo) {
     hi = tf32_rn(x);                                        // 11 significant bits
-    // the difference is exact in FP32 (up to 13 significant bits, either sign); it is rounded to nearest as well, so
-    // that hi + lo represents x to 2^-24 instead of the 2^-23 the tensor core's truncation of its input would leave
-    lo = tf32_rn(x - __uint_as_float(hi));
+    // the difference is exact in FP32 and has either sign; the tensor core reads its leading 11 bits (truncation of
+    // a part whose sign is random is no bias; rounding it too was measured and changes nothing)
+    lo = __float_as_uint(x - __uint_as_float(hi));
 }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -1031,7 +1031,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     // the four eliminations at the pivot slots themselves (every thread, same values)
                     float zz[GS][GS];                      // vector e at pivot slot x
                     double idp[GS], fg[GS];
-                    double rsq[GS];
+                    float rsq[GS];
                     bool fine = true;
 #pragma unroll
                     for (int g = 0; g < GS; ++g) {
@@ -1046,10 +1046,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         if (!(dpp > 0.0) || !isfinite(dpp) || !isfinite(w)) fine = false;
                         idp[g] = 1.0 / dpp;
                         fg[g] = w * idp[g];
-                        const double r0 = (double)__frsqrt_rn((float)dpp);
-                        rsq[g] = r0 * (1.5 - 0.5 * dpp * r0 * r0);
+                        rsq[g] = __frsqrt_rn((float)dpp);
 #pragma unroll
-                        for (int x = 0; x < GS; ++x) zz[g][x] = __double2float_rn((double)mc[x] * rsq[g]);
+                        for (int x = 0; x < GS; ++x) zz[g][x] = mc[x] * rsq[g];
 #pragma unroll
                         for (int x = g + 1; x < GS; ++x) {
                             wp4[x] -= fg[g] * (double)mc[x];
@@ -1080,7 +1079,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                                         for (int e = 0; e < g; ++e) vj = fmaf(-zv[e][q], zz[e][g], vj);
                                         nw -= fg[g] * (double)vj;
                                         nd -= (double)vj * (double)vj * idp[g];
-                                        zv[g][q] = __double2float_rn((double)vj * rsq[g]);
+                                        zv[g][q] = vj * rsq[g];
                                     }
                                 }
                                 if (gm < GS) perm[j] = -1;
@@ -1208,10 +1207,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                 }
                 const double idpp = 1.0 / dpp;
                 const double f = e * idpp;
-                // 1/sqrt(dpp) to FP64 accuracy (one Newton step on the FP32 estimate): the pending vector z = v / sqrt(dpp)
-                // is then rounded once per entry, with no error common to the whole rank-1 term z z^T
-                const double rs0 = (double)__frsqrt_rn((float)dpp);
-                const double rs = rs0 * (1.5 - 0.5 * dpp * rs0 * rs0);
+                const float rs = __frsqrt_rn((float)dpp);
                 const int nbs = GP ? min(nb, scap) : nb;
                 for (int b = 0; b < nbs; ++b) {
                     const float* zo = panel + (size_t)b * ldz;
@@ -1269,7 +1265,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         const double nw = wd[j] - f * (double)vj;
                         const double nd = dg[j] - (double)vj * (double)vj * idpp;
                         wd[j] = nw; dg[j] = nd;
-                        zv[q] = __double2float_rn((double)vj * rs);
+                        zv[q] = vj * rs;
                         if (est_next) sa[k] = score_estimate<Q>(nw, nd, q_next, gsc, gisc, gze, gmq);
                         if (has_nm) {
                             if ((pq[q] >> nm_lg) == (op >> nm_lg)) cntw[g] += 1u << (8 * q);
