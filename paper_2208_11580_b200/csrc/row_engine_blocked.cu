@@ -1250,6 +1250,12 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     const int4 pm = *reinterpret_cast<const int4*>(perm + jb);
                     const int pq[4] = {pm.x, pm.y, pm.z, pm.w};
                     float zv[4];
+                    // the group's FP64 state as 128-bit accesses: a warp's 64-bit accesses at this stride (32 bytes
+                    // between lanes) would meet four to a bank; dead slots keep the value they had
+                    double2* wq = reinterpret_cast<double2*>(wd + jb);
+                    double2* dq = reinterpret_cast<double2*>(dg + jb);
+                    const double2 w01 = wq[0], w23 = wq[1], d01 = dq[0], d23 = dq[1];
+                    double wv[4] = {w01.x, w01.y, w23.x, w23.y}, dv[4] = {d01.x, d01.y, d23.x, d23.y};
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int k = 4 * g + q, j = jb + q;
@@ -1262,9 +1268,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                             continue;
                         }
                         const float vj = c[k] - corr[k];
-                        const double nw = wd[j] - f * (double)vj;
-                        const double nd = dg[j] - (double)vj * (double)vj * idpp;
-                        wd[j] = nw; dg[j] = nd;
+                        const double nw = wv[q] - f * (double)vj;
+                        const double nd = dv[q] - (double)vj * (double)vj * idpp;
+                        wv[q] = nw; dv[q] = nd;
                         zv[q] = vj * rs;
                         if (est_next) sa[k] = score_estimate<Q>(nw, nd, q_next, gsc, gisc, gze, gmq);
                         if (has_nm) {
@@ -1273,6 +1279,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         }
                         if (has_wfull) wfull[pq[q]] = (float)nw;
                     }
+                    wq[0] = make_double2(wv[0], wv[1]); wq[1] = make_double2(wv[2], wv[3]);
+                    dq[0] = make_double2(dv[0], dv[1]); dq[1] = make_double2(dv[2], dv[3]);
                     *reinterpret_cast<float4*>(zb + jb) = make_float4(zv[0], zv[1], zv[2], zv[3]);
                     if (BC && ((live >> (4 * g)) & 0xFu) == 0xFu && jb != (p & ~3)) {
                         // Lemma 1 on the group's own 4 x 4 diagonal block (off-diagonal part; dg holds the diagonal)
@@ -1579,8 +1587,11 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     if (a.d > a.ms) {
         // Shares of rows (equal work per block instead of whole waves): when there are more rows than blocks and they
         // do not divide evenly; not with the N:M pattern or block pruning, whose extra per-row state is not handed over.
-        const bool want_split = a.row_count > blocks && a.row_count % blocks != 0 && a.nm_prune == 0 && !bc &&
-                                !(a.opts.flags & OBC_ENGINE_WHOLE_WAVES);
+        // Only up to three waves: with more, the partly empty last wave is a small part of the launch (and runs faster
+        // than a full one), while rows out of step with each other cost a few per cent on every wave (measured: 5.2 waves
+        // of 3072-column rows 473 -> 469 ms, 10.4 waves of 768-column rows 50 -> 51 ms, 1.4 waves 152 -> 126 ms).
+        const bool want_split = a.row_count > blocks && a.row_count % blocks != 0 && a.row_count < 3 * blocks &&
+                                a.nm_prune == 0 && !bc && !(a.opts.flags & OBC_ENGINE_WHOLE_WAVES);
         const size_t tri = round_up((size_t)blocks * (want_split ? 2 : 1) * a.d * a.cap * sizeof(float), 256);
         const size_t gpan = p.g_vectors ? round_up((size_t)blocks * p.g_vectors * p.g_ld * sizeof(float), 256) : 0;
         const size_t sst = want_split ? round_up((size_t)blocks * blk_split_stride(a.cap), 256) : 0;

@@ -104,3 +104,32 @@ def test_row_shares_prune_trace_quant_replay(threads, d, extra):
                    scale=np.array([float(scale[r].item())]), zero=np.array([float(zero[r].item())]), maxq=14,
                    gpu_codes=gc[r, F][None, :])
     print("row shares", threads, d, rows, {k: v for k, v in st.items() if k not in ("oracle", "trace_rows_max_rel")})
+
+
+@pytest.mark.parametrize("d", [120, 160, 200, 236, 300])
+def test_workspace_query_is_valid_for_every_engine_option(d):
+    """obc_workspace_bytes does not know the options a call will carry: the size it reports must do for every thread
+    count and both engines (row lengths around the on-chip thresholds, which differ by thread count)"""
+    import paper_2208_11580_b200 as m
+    m.load_library()
+    rows = 5
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 6100 + d, "relu")
+    H = oracle.hessian(X).astype(np.float32)
+    ld = (d + 3) // 4 * 4
+    Hinv, info = m.obc_hessian_inverse(_padded(H, ld), DAMP)
+    Wd = _padded(W, ld)
+    ws = torch.empty(m.obc_workspace_bytes(m.OP_PRUNE_TRACE, rows, d), dtype=torch.uint8, device="cuda")
+    ref = None
+    for opts in [(m.ENGINE_BLOCKED, 128, 0), (m.ENGINE_BLOCKED, 256, 0), (m.ENGINE_BLOCKED, 512, 0), (m.ENGINE_BLOCKED, 0, 3),
+                 (m.ENGINE_STREAMING, 0, 0), (m.ENGINE_BLOCKED, 256, 0, m.ENGINE_WHOLE_WAVES)]:
+        order = torch.full((rows, d), -7, dtype=torch.int32, device="cuda")
+        loss = torch.zeros(rows, d, dtype=torch.float32, device="cuda")
+        rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+        m.obc_prune_trace(Wd, Hinv, order, loss, rs, ws=ws, opts=opts)        # raises on OBC_ERR_WORKSPACE
+        torch.cuda.synchronize()
+        assert int(rs.abs().sum()) == 0
+        if ref is None:
+            ref = order.clone()
+            check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy())
+        else:
+            assert (order == ref).float().mean() > 0.99
