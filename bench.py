@@ -443,6 +443,11 @@ def measure(args, name, steps, warmup, rank, world, dev, with_cpu=True, with_e2e
               "flops_model": "2 flops per element of the active lower triangle and deferred update (rank-B update on the tensor "
                              "cores, TF32 m16n8k8); executed = 3 x that: every FP32 operand is split into two TF32 parts and "
                              "three of the four partial products are formed"}
+    if blocked and plan.get("l2_vectors", 0) > 0:
+        tensor["note"] = ("rows this long keep part of their deferred updates in global memory (L2); passes that include those "
+                          "run as FP32 FMAs on the CUDA cores, not on the tensor cores, and are bound by them")
+        tensor["fp32_fma"] = {"achieved": round(tflops, 2), "peak": round(fp32_peak, 1), "unit": "TFLOP/s", "frac": round(tflops / fp32_peak, 4),
+                              "peak_kind": "derived: SMs x 128 FP32 lanes x 2 x max SM clock"}
     # Both engines are reported against HBM.  The streaming engine moves the active triangle once per step.  The blocked
     # engine moves it once per block of deferred updates and applies the block as one rank-B update on the tensor cores;
     # the per-step phase (argmin, pivot column, correction) moves no matrix bytes and is inside the same time.
