@@ -112,14 +112,15 @@ def check_rows(Hinv32, W32, gpu_order, gpu_loss, gpu_w=None, *, mode="prune", sc
 
 
 def record_stats(label, stats):
-    """Appends one line of parity statistics (picks that differ, gaps, errors) to the file named by OBC_PARITY_STATS
-    (default: gpurun_out/parity_stats.jsonl under the repository root) and prints it."""
+    """Prints one line of parity statistics (picks that differ, gaps, errors) and, when the environment variable
+    OBC_PARITY_STATS names a file, appends it there as JSON."""
     rec = {"case": label, **{k: v for k, v in stats.items() if k != "oracle"}}
     print(label, rec)
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    path = os.environ.get("OBC_PARITY_STATS", os.path.join(root, "gpurun_out", "parity_stats.jsonl"))
+    path = os.environ.get("OBC_PARITY_STATS")
+    if not path:
+        return
     try:
-        os.makedirs(os.path.dirname(path), exist_ok=True)
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
         with open(path, "a") as f:
             f.write(json.dumps(rec) + "\n")
     except OSError:
