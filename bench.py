@@ -47,8 +47,10 @@ FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 291.0 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.1 GB moved for 98.1 GB.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.1 / 98.1
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.0 GB moved for 98.13 GB; rows long enough to keep overflow
+# vectors in global memory (d_col > ~2600): profiles/blocked_engine_d3072_rows148_ncu_full.txt, 185.8 GB for 138.33 GB.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.03 / 98.13
+BLOCKED_LONG_TRAFFIC_PER_ALGORITHMIC_BYTE = 185.78 / 138.33
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
@@ -459,9 +461,12 @@ def measure(args, name, steps, warmup, rank, world, dev, with_cpu=True, with_e2e
                 "frac_own_schedule_of_nominal_8TBs": main["frac_of_nominal_8TBs"],
                 "frac_step_by_step_model": round(model_gbs / peak, 3),
                 "frac_step_by_step_model_of_nominal_8TBs": round(model_gbs / NOMINAL_HBM_GBS, 3),
-                "traffic": int(own_bytes / n_eng * BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE) if blocked
+                "traffic": int(own_bytes / n_eng * (BLOCKED_LONG_TRAFFIC_PER_ALGORITHMIC_BYTE if plan.get("l2_vectors", 0) > 0
+                                                    else BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE)) if blocked
                            else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                "traffic_source": ("DRAM bytes, scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes" if blocked else
+                "traffic_source": (("DRAM bytes, scaled from the d=3072 x 148-row ncu capture of this kernel by algorithmic bytes"
+                                    if plan.get("l2_vectors", 0) > 0 else
+                                    "DRAM bytes, scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes") if blocked else
                                    "DRAM bytes, scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
                 "ms_per_launch": round(eng_ms / n_eng, 3), "launches_timed": len(engine_runs),
                 "hbm": main, "tensor" if blocked else "alu": other,
