@@ -133,3 +133,70 @@ def test_workspace_query_is_valid_for_every_engine_option(d):
             check_rows(Hinv.cpu().numpy(), W, order.cpu().numpy(), loss.cpu().numpy())
         else:
             assert (order == ref).float().mean() > 0.99
+
+
+def test_row_shares_partial_trace_and_failing_rows():
+    """rows handed over between blocks with a partial trace (steps < d_col); rows that fail late (a non-finite weight is
+    met when nothing else is left: in the part the second block runs) and early (a replayed order that names a column
+    twice: in the part the first block runs): their status is reported, every other row is unaffected"""
+    import paper_2208_11580_b200 as m
+    m.load_library()
+    raw = m
+    m = WithEngineOpts(raw, raw.ENGINE_BLOCKED, 512, 0)
+    whole = WithEngineOpts(raw, raw.ENGINE_BLOCKED, 512, 0, raw.ENGINE_WHOLE_WAVES)
+    d = 520
+    plan = m.obc_engine_plan(d, False, 0)
+    grid = plan["rows_per_sm"] * plan["sm_count"]
+    rows = grid + grid // 2 + 3
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 7100, "relu")
+    H = oracle.hessian(X).astype(np.float32)
+    ld = (d + 3) // 4 * 4
+    Hinv, info = m.obc_hessian_inverse(_padded(H, ld), DAMP)
+    Hh = Hinv.cpu().numpy()
+    i32 = lambda *s, fill=-7: torch.full(s, fill, dtype=torch.int32, device="cuda")
+    f32 = lambda *s: torch.full(s, -7.0, dtype=torch.float32, device="cuda")
+    sample = np.arange(0, rows, max(1, rows // 20))
+    # ---- partial trace ---------------------------------------------------------------------------------------------
+    steps = d // 3
+    Wd = _padded(W, ld)
+    order, loss, rs = i32(rows, d), f32(rows, d), i32(rows)
+    m.obc_prune_trace(Wd, Hinv, order, loss, rs, steps=steps)
+    o2, l2, r2 = i32(rows, d), f32(rows, d), i32(rows)
+    whole.obc_prune_trace(Wd, Hinv, o2, l2, r2, steps=steps)
+    torch.cuda.synchronize()
+    assert int(rs.abs().sum()) == 0 and int(r2.abs().sum()) == 0
+    o, l = order.cpu().numpy(), loss.cpu().numpy()
+    assert np.all(o[:, steps:] == -7) and np.all(l[:, steps:] == -7.0)
+    check_rows(Hh, W[sample], o[sample], l[sample], steps=steps)
+    assert (o2 == order).float().mean() > 0.995
+    # ---- rows that fail in their last steps ------------------------------------------------------------------------
+    bad = np.array([1, grid // 3, grid, rows - 2])
+    Wb = W.copy()
+    Wb[bad, 7] = np.nan
+    order, loss, rs = i32(rows, d), f32(rows, d), i32(rows)
+    m.obc_prune_trace(_padded(Wb, ld), Hinv, order, loss, rs)
+    torch.cuda.synchronize()
+    st = rs.cpu().numpy()
+    good = np.setdiff1d(np.arange(rows), bad)
+    assert np.all(st[good] == 0) and np.all(st[bad] >= 1)
+    o, l = order.cpu().numpy(), loss.cpu().numpy()
+    for b in bad:
+        assert np.all(o[b, st[b] - 1:] == -1) and np.all(np.isinf(l[b, st[b] - 1:]))
+    gs = good[:: max(1, len(good) // 12)]
+    check_rows(Hh, W[gs], o[gs], l[gs])
+    # ---- rows that fail early in a forced replay (the order names its first column again at step 2) ------------------
+    full_o = torch.from_numpy(o).cuda()
+    full_o[torch.from_numpy(bad).cuda()] = full_o[torch.from_numpy(good[:len(bad)]).cuda()]      # valid orders for those rows
+    bad_o = full_o.clone()
+    bad_o[torch.from_numpy(bad).cuda(), 2] = bad_o[torch.from_numpy(bad).cuda(), 0]
+    counts = torch.full((rows,), d - 40, dtype=torch.int32, device="cuda")
+    out, rsa = f32(rows, d), i32(rows)
+    m.obc_prune_apply(Wd, Hinv, bad_o, counts, out, rsa)
+    ref, rsb = f32(rows, d), i32(rows)
+    whole.obc_prune_apply(Wd, Hinv, full_o, counts, ref, rsb)
+    torch.cuda.synchronize()
+    sa = rsa.cpu().numpy()
+    assert np.all(sa[bad] == 1 + 2) and np.all(sa[good] == 0) and int(rsb.abs().sum()) == 0
+    g, r = out.cpu().numpy()[good], ref.cpu().numpy()[good]
+    wscale = np.abs(W[good]).max(axis=1, keepdims=True)
+    assert (np.abs(g - r) / np.maximum(np.abs(r), wscale)).max() <= 2 * REL_TOL
