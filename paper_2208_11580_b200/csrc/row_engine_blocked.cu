@@ -16,7 +16,8 @@
 // s >= m1, i.e. element (i, j) of the new triangle is read from (max(si, sj), min(si, sj)) of the old one.
 // All such foreign reads come from rows >= m1, which the flush never writes, so it runs in place.
 // The flush is a rank-B update and runs on the tensor cores (warp tiles of 16 rows x 64 columns, TF32 split
-// products, see blk_flush_mma); the pending vectors stay in shared memory.  The O(m) selection state (weights, diagonal) is FP64, as in
+// products, see blk_flush_mma); the pending vectors stay in shared memory (at very long rows further ones sit in a
+// global buffer that stays in L2; the flush reads their operands from there).  The O(m) selection state (weights, diagonal) is FP64, as in
 // the streaming engine.  Once the live triangle fits into the shared memory of the pending vectors, the row
 // finishes on chip with step-by-step updates.
 //
@@ -337,131 +338,10 @@ __device__ __forceinline__ void thread_best(const float (&sa)[KMAX], const doubl
     if (Q && outliers && oslot >= 0) { *s_out = -oe; *slot_out = oslot; *key = float_key(__double2float_rn(-oe)); }
 }
 
-// Applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts
-// it to m1 rows.  srcm[i] = old slot whose data new slot i takes (i itself unless i is a hole).
-// A warp works on tiles of RG rows x 128 columns (row groups dealt out cyclically to the warps); each lane keeps
-// its RG x 4 sub-tile in registers, so RG x 16 bytes per lane are in flight while a tile is fetched and the
-// pending vectors cost RG/4 + 1 shared-memory loads per 4 RG multiply-adds.
-// The first nbs vectors are rows of Z (shared memory, stride ldz), the others rows of G (global memory, stride gld:
-// the overflow part of the pending vectors, small enough to stay in L2).  STREAM: the triangle is far larger than
-// L2 and touched once per flush, so it is loaded and stored with the evict-first hint and leaves L2 to G.
-template <int RG>
-__device__ __forceinline__ void flush_apply_vector(float4 (&acc)[RG], const float* zb, int i0, int j) {
-    const float4 zj = *reinterpret_cast<const float4*>(zb + j);
-#pragma unroll
-    for (int r4 = 0; r4 < RG / 4; ++r4) {
-        const float4 za = *reinterpret_cast<const float4*>(zb + i0 + 4 * r4);
-        const float zi[4] = {za.x, za.y, za.z, za.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float4& t = acc[4 * r4 + q];
-            t.x = fmaf(-zi[q], zj.x, t.x);
-            t.y = fmaf(-zi[q], zj.y, t.y);
-            t.z = fmaf(-zi[q], zj.z, t.z);
-            t.w = fmaf(-zi[q], zj.w, t.w);
-        }
-    }
-}
-
-// Same with the column operand already in registers and the row operand in a small shared-memory block
-// (zrow[0..RG)): used for the overflow vectors, whose column operands are prefetched from L2.
-template <int RG>
-__device__ __forceinline__ void flush_apply_staged(float4 (&acc)[RG], const float4 zj, const float* zrow) {
-#pragma unroll
-    for (int r4 = 0; r4 < RG / 4; ++r4) {
-        const float4 za = *reinterpret_cast<const float4*>(zrow + 4 * r4);
-        const float zi[4] = {za.x, za.y, za.z, za.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float4& t = acc[4 * r4 + q];
-            t.x = fmaf(-zi[q], zj.x, t.x);
-            t.y = fmaf(-zi[q], zj.y, t.y);
-            t.z = fmaf(-zi[q], zj.z, t.z);
-            t.w = fmaf(-zi[q], zj.w, t.w);
-        }
-    }
-}
-
-// zstage: per-warp staging block of (nb - nbs) x RG floats for the row operands of the overflow vectors.
-template <int NT, int RG, bool STREAM>
-__device__ __forceinline__ void blk_flush(float* __restrict__ Hp, int ldp, int m1, int nb, int nbs, const float* Z,
-                                          int ldz, const float* G, int gld, float* zstage, const unsigned short* srcm,
-                                          const uint32_t* colmask) {
-    constexpr int NW = NT / 32;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nrg = (m1 + RG - 1) / RG;
-    for (int rg = warp; rg < nrg; rg += NW) {
-        const int i0 = rg * RG;
-        const int nrows = min(RG, m1 - i0);
-        int sr[RG];
-#pragma unroll
-        for (int r = 0; r < RG; ++r) sr[r] = (r < nrows) ? (int)srcm[i0 + r] : i0;
-        const int jend = i0 + nrows;                           // columns [0, jend) hold data of this row group
-        const int nbg = nb - nbs;
-        if (nbg > 0) {                                         // row operands of the overflow vectors -> staging block
-            __syncwarp();
-            for (int e = lane; e < nbg * (RG / 4); e += 32) {
-                const int v = e / (RG / 4), q = e - v * (RG / 4);
-                *reinterpret_cast<float4*>(zstage + v * RG + 4 * q) =
-                    *reinterpret_cast<const float4*>(G + (size_t)v * gld + i0 + 4 * q);
-            }
-            __syncwarp();
-        }
-        for (int c0 = 0; c0 < jend; c0 += 128) {
-            const int j = c0 + (lane << 2);
-            if (j >= jend) continue;                           // whole float4 above the diagonal of every row
-            float4 acc[RG];
-#pragma unroll
-            for (int r = 0; r < RG; ++r) {
-                acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (r < nrows && j <= i0 + r) {
-                    const float4* src = reinterpret_cast<const float4*>(Hp + (size_t)sr[r] * ldp + j);
-                    acc[r] = STREAM ? __ldcs(src) : *src;
-                }
-            }
-            // columns of this lane that are holes: their data sits in the mover's row
-            const uint32_t my4 = (colmask[j >> 5] >> (j & 31)) & 0xFu;
-            if (my4) {
-#pragma unroll
-                for (int comp = 0; comp < 4; ++comp) {
-                    if (!((my4 >> comp) & 1u)) continue;
-                    const int jj = j + comp;
-                    const int sj = (int)srcm[jj];
-#pragma unroll
-                    for (int r = 0; r < RG; ++r) {
-                        if (r < nrows && jj <= i0 + r) {
-                            const int hi = max(sr[r], sj), lo = min(sr[r], sj);
-                            const float val = Hp[(size_t)hi * ldp + lo];
-                            if (comp == 0) acc[r].x = val; else if (comp == 1) acc[r].y = val;
-                            else if (comp == 2) acc[r].z = val; else acc[r].w = val;
-                        }
-                    }
-                }
-            }
-            for (int b = 0; b < nbs; ++b) flush_apply_vector<RG>(acc, Z + (size_t)b * ldz, i0, j);
-            if (nbg > 0) {                                     // column operands from L2, two vectors ahead
-                const float* gj = G + j;
-                float4 q0 = *reinterpret_cast<const float4*>(gj), q1 = q0;
-                if (nbg > 1) q1 = *reinterpret_cast<const float4*>(gj + gld);
-                for (int b = 0; b < nbg; b += 2) {
-                    float4 n0 = q0, n1 = q1;
-                    if (b + 2 < nbg) n0 = *reinterpret_cast<const float4*>(gj + (size_t)(b + 2) * gld);
-                    if (b + 3 < nbg) n1 = *reinterpret_cast<const float4*>(gj + (size_t)(b + 3) * gld);
-                    flush_apply_staged<RG>(acc, q0, zstage + b * RG);
-                    if (b + 1 < nbg) flush_apply_staged<RG>(acc, q1, zstage + (b + 1) * RG);
-                    q0 = n0; q1 = n1;
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < RG; ++r)
-                if (r < nrows && j <= i0 + r) {
-                    float4* dst = reinterpret_cast<float4*>(Hp + (size_t)(i0 + r) * ldp + j);
-                    if (STREAM) __stcs(dst, acc[r]); else *dst = acc[r];
-                }
-        }
-    }
-}
-
+// The flush applies the nb pending vectors Z[b][.] (already in the new slot numbering) to the triangle and compacts it
+// to m1 rows.  srcm[i] = old slot whose data new slot i takes (i itself unless i is a hole).  The triangle is far
+// larger than L2 and touched once per flush, so it is loaded and stored with the evict-first hint and leaves L2 to
+// the overflow part of the pending vectors.
 // ---- flush on the tensor cores -----------------------------------------------------------------------------------
 // The flush is a rank-nb update, H -= Z^T Z with nb <= 64: a dense contraction.  A warp takes tiles of 16 rows x
 // 64 columns; the increment of a tile is formed by mma.sync m16n8k8 (TF32 inputs, FP32 accumulation over 8 pending
@@ -488,14 +368,33 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int NT, bool STREAM>
-__device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, int m1, int nb, const float* Z, int ldz,
+// GP: pending vectors nbs .. nb - 1 are rows of G (global memory, stride gld: the overflow part, resident in L2).  Their
+// row operands are copied once per row group into the warp's staging block zstage (16 floats per vector); their column
+// operands are read from L2 in the fragment layout, 8 vectors at a time.
+// first product of a chain: the accumulator operand is zero
+__device__ __forceinline__ void mma_tf32_z(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+// two values at once: the integer part of the split per value, the subtraction as one packed FP32 instruction
+__device__ __forceinline__ void tf32_split2(float2 x, uint32_t& hi0, uint32_t& hi1, uint32_t& lo0, uint32_t& lo1) {
+    hi0 = tf32_rn(x.x); hi1 = tf32_rn(x.y);
+    const float2 l = __ffma2_rn(make_float2(__uint_as_float(hi0), __uint_as_float(hi1)), make_float2(-1.f, -1.f), x);
+    lo0 = __float_as_uint(l.x); lo1 = __float_as_uint(l.y);
+}
+
+template <int NT, bool STREAM, bool GP>
+__device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, int m1, int nb, int nbs, const float* Z, int ldz,
+                                              const float* __restrict__ G, int gld, float* zstage,
                                               const unsigned short* srcm, const uint32_t* colmask) {
     constexpr int NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int nrg = (m1 + 15) >> 4;
-    const int ksteps = (nb + 7) >> 3;
+    const int ksteps = ((GP ? nbs : nb) + 7) >> 3;
+    const int nbg = GP ? nb - nbs : 0;
+    const int ksteps_g = (nbg + 7) >> 3;
     // The products are cheap next to the latency of memory, and a warp has one tile (4 KB) in registers at a time:
     // a cursor runs FLUSH_AHEAD tiles ahead of the warp through its sequence of tiles and pulls them into L2
     // (measured at d_col = 2304: 12 % off the pass with a distance of 1 or 2 tiles, less with 4, a loss from 8 on).
@@ -517,6 +416,15 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
         const int rr[2] = {i0 + g, i0 + g + 8};                // the lane's two rows
         const bool in[2] = {rr[0] < m1, rr[1] < m1};
         const int sr[2] = {in[0] ? (int)srcm[rr[0]] : 0, in[1] ? (int)srcm[rr[1]] : 0};
+        if (GP && nbg > 0) {                                   // row operands of the overflow vectors -> staging block
+            __syncwarp();
+            for (int e = lane; e < nbg * 4; e += 32) {
+                const int v = e >> 2, q = e & 3;
+                *reinterpret_cast<float4*>(zstage + v * 16 + 4 * q) =
+                    *reinterpret_cast<const float4*>(G + (size_t)v * gld + i0 + 4 * q);
+            }
+            __syncwarp();
+        }
         for (int c0 = 0; c0 < jend; c0 += 64) {
             const int ngroups = min(4, (jend - c0 + 15) >> 4);
             prefetch_next();
@@ -524,27 +432,48 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
             float acc[8][4];
 #pragma unroll
             for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
-            for (int ks = 0; ks < ksteps; ++ks) {
-                const int k0 = (ks << 3) + t, k1 = k0 + 4;
-                const float* z0 = Z + (size_t)k0 * ldz;
-                const float* z1 = Z + (size_t)k1 * ldz;
-                const bool v0 = k0 < nb, v1 = k1 < nb;
+            for (int ks = 0; ks < ksteps + ksteps_g; ++ks) {
+                const bool from_g = GP && ks >= ksteps;
+                const int k0 = ((from_g ? ks - ksteps : ks) << 3) + t, k1 = k0 + 4;
+                const bool v0 = k0 < (from_g ? nbg : (GP ? nbs : nb)), v1 = k1 < (from_g ? nbg : (GP ? nbs : nb));
                 uint32_t ah[4], al[4];
-                tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
-                tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
-                tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
-                tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
                 uint32_t bh[8][2], bl[8][2];                              // the 8 MMA tiles: (k0, k1) parts
+                if (!from_g) {
+                    const float* z0 = Z + (size_t)k0 * ldz;
+                    const float* z1 = Z + (size_t)k1 * ldz;
+                    tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
+                    tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
+                    tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
+                    tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
-                    float2 b0 = make_float2(0.f, 0.f), b1 = b0;           // (a group past the end multiplies zeros)
-                    if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
-                    if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
-                    tf32_split(b0.x, bh[2 * u][0], bl[2 * u][0]);
-                    tf32_split(b1.x, bh[2 * u][1], bl[2 * u][1]);
-                    tf32_split(b0.y, bh[2 * u + 1][0], bl[2 * u + 1][0]);
-                    tf32_split(b1.y, bh[2 * u + 1][1], bl[2 * u + 1][1]);
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
+                        float2 b0 = make_float2(0.f, 0.f), b1 = b0;           // (a group past the end multiplies zeros)
+                        if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
+                        if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
+                        tf32_split2(b0, bh[2 * u][0], bh[2 * u + 1][0], bl[2 * u][0], bl[2 * u + 1][0]);
+                        tf32_split2(b1, bh[2 * u][1], bh[2 * u + 1][1], bl[2 * u][1], bl[2 * u + 1][1]);
+                    }
+                } else {
+                    const float* z0 = G + (size_t)k0 * gld;
+                    const float* z1 = G + (size_t)k1 * gld;
+                    float2 b0[4], b1[4];                                      // all loads of the step in flight together
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = c0 + (u << 4) + (g << 1);               // < round_up(m1, 16) <= gld
+                        b0[u] = make_float2(0.f, 0.f); b1[u] = b0[u];
+                        if (u < ngroups && v0) b0[u] = *reinterpret_cast<const float2*>(z0 + c);
+                        if (u < ngroups && v1) b1[u] = *reinterpret_cast<const float2*>(z1 + c);
+                    }
+                    tf32_split(v0 ? zstage[k0 * 16 + g] : 0.f, ah[0], al[0]);      // (rows past m1 are never stored)
+                    tf32_split(v0 ? zstage[k0 * 16 + g + 8] : 0.f, ah[1], al[1]);
+                    tf32_split(v1 ? zstage[k1 * 16 + g] : 0.f, ah[2], al[2]);
+                    tf32_split(v1 ? zstage[k1 * 16 + g + 8] : 0.f, ah[3], al[3]);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        tf32_split2(b0[u], bh[2 * u][0], bh[2 * u + 1][0], bl[2 * u][0], bl[2 * u + 1][0]);
+                        tf32_split2(b1[u], bh[2 * u][1], bh[2 * u + 1][1], bl[2 * u][1], bl[2 * u + 1][1]);
+                    }
                 }
                 // The tensor core rounds every result toward zero (measured: the products of one instruction are
                 // summed with guard bits, then truncated to FP32).  On a running accumulator that is a bias of about
@@ -555,9 +484,7 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                 // products after the previous one into it: their latency is long.
                 float dk[8][4];
 #pragma unroll
-                for (int n = 0; n < 8; ++n) { dk[n][0] = 0.f; dk[n][1] = 0.f; dk[n][2] = 0.f; dk[n][3] = 0.f; }
-#pragma unroll
-                for (int n = 0; n < 8; ++n) mma_tf32(dk[n], al, bh[n][0], bh[n][1]);
+                for (int n = 0; n < 8; ++n) mma_tf32_z(dk[n], al, bh[n][0], bh[n][1]);
 #pragma unroll
                 for (int n = 0; n < 8; ++n) mma_tf32(dk[n], ah, bl[n][0], bl[n][1]);
 #pragma unroll
@@ -570,7 +497,12 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
 #pragma unroll
                 for (int n = 0; n < 8; ++n)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[n][e] += __uint_as_float(__float_as_uint(dk[n][e]) | 1u);
+                    for (int e = 0; e < 4; e += 2) {                     // (two additions per instruction)
+                        const float2 r = __fadd2_rn(make_float2(acc[n][e], acc[n][e + 1]),
+                                                    make_float2(__uint_as_float(__float_as_uint(dk[n][e]) | 1u),
+                                                                __uint_as_float(__float_as_uint(dk[n][e + 1]) | 1u)));
+                        acc[n][e] = r.x; acc[n][e + 1] = r.y;
+                    }
             }
             // ---- the tile of H (in L2 by now: the cursor passed it two tiles ago), minus the increment -----------
             float4 hv[4][2];
@@ -892,10 +824,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                         atomicOr(&colmask[h >> 5], 1u << (h & 31));
                     }
                     __syncthreads();
-                    if (!GP || nb <= scap)
-                        blk_flush_mma<NT, true>(HP, ldp, m1, nb, panel, ldz, srcm, colmask);      // evict-first at every row length (~1 %)
+                    if (!GP)
+                        blk_flush_mma<NT, true, false>(HP, ldp, m1, nb, nb, panel, ldz, nullptr, 0, nullptr, srcm, colmask);      // evict-first at every row length (~1 %)
                     else
-                        blk_flush<NT, 16, (NT >= 512)>(HP, ldp, m1, nb, min(nb, scap), panel, ldz, GVEC, gld, ZSTAGE, srcm, colmask);
+                        blk_flush_mma<NT, true, true>(HP, ldp, m1, nb, min(nb, scap), panel, ldz, GVEC, gld, ZSTAGE, srcm, colmask);
                     __syncthreads();
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
@@ -1445,16 +1377,17 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     p.smem = share;
     p.panel_floats = (int)((share - fixed) / 4);
     p.ms = blk_pick_ms(d, share - fixed);
-    // Very long rows (d_col > ~2600): shared memory holds fewer than 16 pending vectors and the flush is bound by
-    // the traffic of the triangle; further vectors go to a global buffer small enough to stay in L2 (the triangle
-    // itself is streamed past it with evict-first hints).  Measured at d_col = 3072: 99 -> 83 ms per wave of rows;
-    // at 2304 (19 vectors in shared memory) it gains nothing, so it is not used there.
+    // Very long rows (d_col > ~2600): shared memory holds fewer than 16 pending vectors, so a pass over the triangle
+    // applies few updates; further vectors go to a global buffer small enough to stay in L2 (the triangle itself is
+    // streamed past it with evict-first hints).  Measured at d_col = 3072: 99 -> 80 ms per wave of rows; at 2304
+    // (19 vectors in shared memory) it gains nothing, so it is not used there.
     p.g_ld = (cap + 15) & ~15;
     p.g_vectors = 0;
     if (p.nt == 512) {
         const int in_smem = p.panel_floats / blk_ldz(cap);
         int g = (int)(BLK_L2_PANEL_BUDGET / ((size_t)di.sm_count * p.g_ld * 4));
         if (g > 32) g = 32;
+        g &= ~7;                                                   // the flush multiplies 8 vectors at a time
         const size_t stage = (size_t)(p.nt / 32) * g * 16 * 4;     // per-warp staging of their row operands
         if (in_smem < 16 && g >= 4 && share - fixed >= stage + 4 * min_panel) {
             p.g_vectors = g;
