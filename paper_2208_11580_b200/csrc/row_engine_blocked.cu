@@ -432,48 +432,16 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
             float acc[8][4];
 #pragma unroll
             for (int n = 0; n < 8; ++n) { acc[n][0] = 0.f; acc[n][1] = 0.f; acc[n][2] = 0.f; acc[n][3] = 0.f; }
-            for (int ks = 0; ks < ksteps + ksteps_g; ++ks) {
-                const bool from_g = GP && ks >= ksteps;
-                const int k0 = ((from_g ? ks - ksteps : ks) << 3) + t, k1 = k0 + 4;
-                const bool v0 = k0 < (from_g ? nbg : (GP ? nbs : nb)), v1 = k1 < (from_g ? nbg : (GP ? nbs : nb));
+            // one step: 8 pending vectors (this lane: vectors k0 = 8 ks + t and k0 + 4) times the tile's rows and columns
+            auto kstep = [&](const float (&av)[4], const float2 (&b0)[4], const float2 (&b1)[4]) {
                 uint32_t ah[4], al[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tf32_split(av[q], ah[q], al[q]);
                 uint32_t bh[8][2], bl[8][2];                              // the 8 MMA tiles: (k0, k1) parts
-                if (!from_g) {
-                    const float* z0 = Z + (size_t)k0 * ldz;
-                    const float* z1 = Z + (size_t)k1 * ldz;
-                    tf32_split(v0 && in[0] ? z0[rr[0]] : 0.f, ah[0], al[0]);
-                    tf32_split(v0 && in[1] ? z0[rr[1]] : 0.f, ah[1], al[1]);
-                    tf32_split(v1 && in[0] ? z1[rr[0]] : 0.f, ah[2], al[2]);
-                    tf32_split(v1 && in[1] ? z1[rr[1]] : 0.f, ah[3], al[3]);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
-                        float2 b0 = make_float2(0.f, 0.f), b1 = b0;           // (a group past the end multiplies zeros)
-                        if (u < ngroups && v0) b0 = *reinterpret_cast<const float2*>(z0 + c);
-                        if (u < ngroups && v1) b1 = *reinterpret_cast<const float2*>(z1 + c);
-                        tf32_split2(b0, bh[2 * u][0], bh[2 * u + 1][0], bl[2 * u][0], bl[2 * u + 1][0]);
-                        tf32_split2(b1, bh[2 * u][1], bh[2 * u + 1][1], bl[2 * u][1], bl[2 * u + 1][1]);
-                    }
-                } else {
-                    const float* z0 = G + (size_t)k0 * gld;
-                    const float* z1 = G + (size_t)k1 * gld;
-                    float2 b0[4], b1[4];                                      // all loads of the step in flight together
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int c = c0 + (u << 4) + (g << 1);               // < round_up(m1, 16) <= gld
-                        b0[u] = make_float2(0.f, 0.f); b1[u] = b0[u];
-                        if (u < ngroups && v0) b0[u] = *reinterpret_cast<const float2*>(z0 + c);
-                        if (u < ngroups && v1) b1[u] = *reinterpret_cast<const float2*>(z1 + c);
-                    }
-                    tf32_split(v0 ? zstage[k0 * 16 + g] : 0.f, ah[0], al[0]);      // (rows past m1 are never stored)
-                    tf32_split(v0 ? zstage[k0 * 16 + g + 8] : 0.f, ah[1], al[1]);
-                    tf32_split(v1 ? zstage[k1 * 16 + g] : 0.f, ah[2], al[2]);
-                    tf32_split(v1 ? zstage[k1 * 16 + g + 8] : 0.f, ah[3], al[3]);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        tf32_split2(b0[u], bh[2 * u][0], bh[2 * u + 1][0], bl[2 * u][0], bl[2 * u + 1][0]);
-                        tf32_split2(b1[u], bh[2 * u][1], bh[2 * u + 1][1], bl[2 * u][1], bl[2 * u + 1][1]);
-                    }
+                for (int u = 0; u < 4; ++u) {
+                    tf32_split2(b0[u], bh[2 * u][0], bh[2 * u + 1][0], bl[2 * u][0], bl[2 * u + 1][0]);
+                    tf32_split2(b1[u], bh[2 * u][1], bh[2 * u + 1][1], bl[2 * u][1], bl[2 * u + 1][1]);
                 }
                 // The tensor core rounds every result toward zero (measured: the products of one instruction are
                 // summed with guard bits, then truncated to FP32).  On a running accumulator that is a bias of about
@@ -503,6 +471,47 @@ __device__ __forceinline__ void blk_flush_mma(float* __restrict__ Hp, int ldp, i
                                                                 __uint_as_float(__float_as_uint(dk[n][e + 1]) | 1u)));
                         acc[n][e] = r.x; acc[n][e + 1] = r.y;
                     }
+            };
+            // column operands of an overflow step, straight from L2; issued one step ahead of their use
+            float2 pb0[4], pb1[4];
+            auto load_g = [&](int kg) {
+                const int k0 = (kg << 3) + t, k1 = k0 + 4;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + (u << 4) + (g << 1);               // < round_up(m1, 16) <= gld
+                    pb0[u] = make_float2(0.f, 0.f); pb1[u] = pb0[u];
+                    if (u < ngroups && k0 < nbg) pb0[u] = *reinterpret_cast<const float2*>(G + (size_t)k0 * gld + c);
+                    if (u < ngroups && k1 < nbg) pb1[u] = *reinterpret_cast<const float2*>(G + (size_t)k1 * gld + c);
+                }
+            };
+            if (GP && ksteps_g > 0) load_g(0);                            // in flight during the shared-memory steps
+            for (int ks = 0; ks < ksteps; ++ks) {
+                const int k0 = (ks << 3) + t, k1 = k0 + 4;
+                const bool v0 = k0 < (GP ? nbs : nb), v1 = k1 < (GP ? nbs : nb);
+                const float* z0 = Z + (size_t)k0 * ldz;
+                const float* z1 = Z + (size_t)k1 * ldz;
+                const float av[4] = {v0 && in[0] ? z0[rr[0]] : 0.f, v0 && in[1] ? z0[rr[1]] : 0.f,
+                                     v1 && in[0] ? z1[rr[0]] : 0.f, v1 && in[1] ? z1[rr[1]] : 0.f};
+                float2 b0[4], b1[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + (u << 4) + (g << 1);               // < m1 + 16 <= ldz
+                    b0[u] = make_float2(0.f, 0.f); b1[u] = b0[u];         // (a group past the end multiplies zeros)
+                    if (u < ngroups && v0) b0[u] = *reinterpret_cast<const float2*>(z0 + c);
+                    if (u < ngroups && v1) b1[u] = *reinterpret_cast<const float2*>(z1 + c);
+                }
+                kstep(av, b0, b1);
+            }
+            if (GP) for (int kg = 0; kg < ksteps_g; ++kg) {
+                const int k0 = (kg << 3) + t, k1 = k0 + 4;
+                const bool v0 = k0 < nbg, v1 = k1 < nbg;
+                const float av[4] = {v0 ? zstage[k0 * 16 + g] : 0.f, v0 ? zstage[k0 * 16 + g + 8] : 0.f,      // (rows past m1
+                                     v1 ? zstage[k1 * 16 + g] : 0.f, v1 ? zstage[k1 * 16 + g + 8] : 0.f};     // are never stored)
+                float2 b0[4], b1[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { b0[u] = pb0[u]; b1[u] = pb1[u]; }
+                if (kg + 1 < ksteps_g) load_g(kg + 1);
+                kstep(av, b0, b1);
             }
             // ---- the tile of H (in L2 by now: the cursor passed it two tiles ago), minus the increment -----------
             float4 hv[4][2];
@@ -1377,19 +1386,20 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     p.smem = share;
     p.panel_floats = (int)((share - fixed) / 4);
     p.ms = blk_pick_ms(d, share - fixed);
-    // Very long rows (d_col > ~2600): shared memory holds fewer than 16 pending vectors, so a pass over the triangle
+    // Long rows (d_col > ~1900): shared memory holds fewer than 24 pending vectors, so a pass over the triangle
     // applies few updates; further vectors go to a global buffer small enough to stay in L2 (the triangle itself is
-    // streamed past it with evict-first hints).  Measured at d_col = 3072: 99 -> 80 ms per wave of rows; at 2304
-    // (19 vectors in shared memory) it gains nothing, so it is not used there.
+    // streamed past it with evict-first hints).  Measured per wave of rows: d_col = 3072 (14 vectors in shared
+    // memory + 24) 99 -> 73 ms; d_col = 2304 (19 + 16) 37.0 -> 36.3 ms, with 8 or 32 more no gain there.
     p.g_ld = (cap + 15) & ~15;
     p.g_vectors = 0;
     if (p.nt == 512) {
         const int in_smem = p.panel_floats / blk_ldz(cap);
         int g = (int)(BLK_L2_PANEL_BUDGET / ((size_t)di.sm_count * p.g_ld * 4));
         if (g > 32) g = 32;
+        if (in_smem >= 16 && g > 16) g = 16;
         g &= ~7;                                                   // the flush multiplies 8 vectors at a time
         const size_t stage = (size_t)(p.nt / 32) * g * 16 * 4;     // per-warp staging of their row operands
-        if (in_smem < 16 && g >= 4 && share - fixed >= stage + 4 * min_panel) {
+        if (in_smem < 24 && g >= 8 && share - fixed >= stage + 4 * min_panel) {
             p.g_vectors = g;
             p.panel_floats = (int)((share - fixed - stage) / 4);
             p.ms = blk_pick_ms(d, share - fixed - stage);
