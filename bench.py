@@ -46,11 +46,11 @@ FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # profiles/streaming_engine_d1152_rows148_ncu_full.txt (291.0 GB moved for 603.3 GB of 8 m^2 model bytes); the
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 291.0 / 603.3
-# The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), from
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.0 GB moved for 98.13 GB; rows long enough to keep overflow
-# vectors in global memory (d_col > ~2600): profiles/blocked_engine_d3072_rows148_ncu_full.txt, 185.8 GB for 138.33 GB.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = 120.03 / 98.13
-BLOCKED_LONG_TRAFFIC_PER_ALGORITHMIC_BYTE = 185.78 / 138.33
+# The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), per captured row length:
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 86.34 GB moved for 62.21 GB;
+# profiles/blocked_engine_d3072_rows148_ncu_full.txt: 201.79 GB for 147.73 GB.  Other row lengths run other
+# configurations of the kernel (threads per row, pending vectors in L2) and have no capture: traffic is null there.
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = {2304: 86.34 / 62.21, 3072: 201.79 / 147.73}
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:
@@ -446,10 +446,8 @@ def measure(args, name, steps, warmup, rank, world, dev, with_cpu=True, with_e2e
                              "cores, TF32 m16n8k8); executed = 3 x that: every FP32 operand is split into two TF32 parts and "
                              "three of the four partial products are formed"}
     if blocked and plan.get("l2_vectors", 0) > 0:
-        tensor["note"] = ("rows this long keep part of their deferred updates in global memory (L2); passes that include those "
-                          "run as FP32 FMAs on the CUDA cores, not on the tensor cores, and are bound by them")
-        tensor["fp32_fma"] = {"achieved": round(tflops, 2), "peak": round(fp32_peak, 1), "unit": "TFLOP/s", "frac": round(tflops / fp32_peak, 4),
-                              "peak_kind": "derived: SMs x 128 FP32 lanes x 2 x max SM clock"}
+        tensor["note"] = ("rows this long keep %d of their deferred updates per pass in global memory (resident in L2); the rank-B "
+                          "update reads their operands from there in the MMA fragment layout" % plan["l2_vectors"])
     # Both engines are reported against HBM.  The streaming engine moves the active triangle once per step.  The blocked
     # engine moves it once per block of deferred updates and applies the block as one rank-B update on the tensor cores;
     # the per-step phase (argmin, pivot column, correction) moves no matrix bytes and is inside the same time.
@@ -461,12 +459,12 @@ def measure(args, name, steps, warmup, rank, world, dev, with_cpu=True, with_e2e
                 "frac_own_schedule_of_nominal_8TBs": main["frac_of_nominal_8TBs"],
                 "frac_step_by_step_model": round(model_gbs / peak, 3),
                 "frac_step_by_step_model_of_nominal_8TBs": round(model_gbs / NOMINAL_HBM_GBS, 3),
-                "traffic": int(own_bytes / n_eng * (BLOCKED_LONG_TRAFFIC_PER_ALGORITHMIC_BYTE if plan.get("l2_vectors", 0) > 0
-                                                    else BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE)) if blocked
+                "traffic": (int(own_bytes / n_eng * BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE[layer.d])
+                            if layer.d in BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE else None) if blocked
                            else int(model_bytes / n_eng * ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                "traffic_source": (("DRAM bytes, scaled from the d=3072 x 148-row ncu capture of this kernel by algorithmic bytes"
-                                    if plan.get("l2_vectors", 0) > 0 else
-                                    "DRAM bytes, scaled from the d=2304 x 148-row ncu capture of this kernel by algorithmic bytes") if blocked else
+                "traffic_source": (("DRAM bytes, scaled from the d=%d x 148-row ncu capture of this kernel by algorithmic bytes" % layer.d
+                                    if layer.d in BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE else
+                                    "no ncu capture of the kernel configuration this row length runs") if blocked else
                                    "DRAM bytes, scaled from the d=1152 x 148-row ncu capture by algorithmic bytes"),
                 "ms_per_launch": round(eng_ms / n_eng, 3), "launches_timed": len(engine_runs),
                 "hbm": main, "tensor" if blocked else "alu": other,

@@ -1386,20 +1386,20 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     p.smem = share;
     p.panel_floats = (int)((share - fixed) / 4);
     p.ms = blk_pick_ms(d, share - fixed);
-    // Long rows (d_col > ~1900): shared memory holds fewer than 24 pending vectors, so a pass over the triangle
+    // Very long rows (d_col > ~2600): shared memory holds fewer than 16 pending vectors, so a pass over the triangle
     // applies few updates; further vectors go to a global buffer small enough to stay in L2 (the triangle itself is
-    // streamed past it with evict-first hints).  Measured per wave of rows: d_col = 3072 (14 vectors in shared
-    // memory + 24) 99 -> 73 ms; d_col = 2304 (19 + 16) 37.0 -> 36.3 ms, with 8 or 32 more no gain there.
+    // streamed past it with evict-first hints).  Measured at d_col = 3072: 99 -> 73 ms per wave of rows.  At 2304 (19
+    // vectors in shared memory) 16 more gain 2 % on one wave of rows and lose 2 % when rows are handed over between
+    // blocks (rows out of step with each other compete for L2), so it is not used there.
     p.g_ld = (cap + 15) & ~15;
     p.g_vectors = 0;
     if (p.nt == 512) {
         const int in_smem = p.panel_floats / blk_ldz(cap);
         int g = (int)(BLK_L2_PANEL_BUDGET / ((size_t)di.sm_count * p.g_ld * 4));
         if (g > 32) g = 32;
-        if (in_smem >= 16 && g > 16) g = 16;
         g &= ~7;                                                   // the flush multiplies 8 vectors at a time
         const size_t stage = (size_t)(p.nt / 32) * g * 16 * 4;     // per-warp staging of their row operands
-        if (in_smem < 24 && g >= 8 && share - fixed >= stage + 4 * min_panel) {
+        if (in_smem < 16 && g >= 8 && share - fixed >= stage + 4 * min_panel) {
             p.g_vectors = g;
             p.panel_floats = (int)((share - fixed - stage) / 4);
             p.ms = blk_pick_ms(d, share - fixed - stage);
