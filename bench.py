@@ -47,10 +47,10 @@ FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # traffic of a full-size launch is scaled from it by the algorithmic bytes (traffic grows with them).
 ENGINE_TRAFFIC_PER_ALGORITHMIC_BYTE = 291.0 / 603.3
 # The same for the blocked engine, relative to ITS algorithmic bytes (blocked_bytes_flops), per captured row length:
-# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 86.34 GB moved for 62.21 GB;
+# profiles/blocked_engine_d2304_rows148_ncu_full.txt: 120.04 GB moved for 98.13 GB;
 # profiles/blocked_engine_d3072_rows148_ncu_full.txt: 201.79 GB for 147.73 GB.  Other row lengths run other
 # configurations of the kernel (threads per row, pending vectors in L2) and have no capture: traffic is null there.
-BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = {2304: 86.34 / 62.21, 3072: 201.79 / 147.73}
+BLOCKED_TRAFFIC_PER_ALGORITHMIC_BYTE = {2304: 120.04 / 98.13, 3072: 201.79 / 147.73}
 
 
 def model_bytes_full(d: int, first: int | None = None, steps: int | None = None) -> int:

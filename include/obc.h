@@ -85,10 +85,11 @@ unsigned long long obc_kernel_launches(void);
  *   threads     : BLOCKED engine, threads per row: 128, 256, 512, or 0 = chosen from d_col and row_count.
  *   max_pending : BLOCKED engine, upper limit on the number of deferred updates, 1..64, or 0 = as many as the
  *                 shared memory holds.
- *   flags       : OBC_ENGINE_WHOLE_WAVES or 0.  By default, when a call has more rows than the GPU holds at once (up to
- *                 three times as many) and they do not divide evenly, the BLOCKED engine gives every thread block the same amount of work, so a
- *                 row may be started by one block and finished by another; with OBC_ENGINE_WHOLE_WAVES every row stays
- *                 on one block and the last wave runs partly empty.
+ *   flags       : OBC_ENGINE_WHOLE_WAVES or 0.  By default, when a call has more rows than the GPU holds at once (with
+ *                 several rows per SM: up to three times as many) and they do not divide evenly, the BLOCKED engine
+ *                 gives every thread block the same amount of work, so a row may be started by one block and finished
+ *                 by another; with OBC_ENGINE_WHOLE_WAVES every row stays on one block and the last wave runs partly
+ *                 empty.
  * Values outside these sets make the call return OBC_ERR_INVALID_ARG.  Workspace sizes reported by
  * obc_workspace_bytes are valid for every choice. */
 typedef struct {

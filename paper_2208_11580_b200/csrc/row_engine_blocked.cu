@@ -1530,10 +1530,13 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     if (a.d > a.ms) {
         // Shares of rows (equal work per block instead of whole waves): when there are more rows than blocks and they
         // do not divide evenly; not with the N:M pattern or block pruning, whose extra per-row state is not handed over.
-        // Only up to three waves: with more, the partly empty last wave is a small part of the launch (and runs faster
-        // than a full one), while rows out of step with each other cost a few per cent on every wave (measured: 5.2 waves
-        // of 3072-column rows 473 -> 469 ms, 10.4 waves of 768-column rows 50 -> 51 ms, 1.4 waves 152 -> 126 ms).
-        const bool want_split = a.row_count > blocks && a.row_count % blocks != 0 && a.row_count < 3 * blocks &&
+        // With one row per SM (long rows) at any number of waves: measured 5.2 waves of 3072-column rows 428 -> 385 ms,
+        // 10.1 waves 794 -> 757 ms, 5.2 waves of 2304-column rows 219 -> 194 ms, of 1536-column rows 75.8 -> 68.7 ms.
+        // With several rows per SM only up to three waves: the pieces are smaller and the kernels with this code slower,
+        // above all the forced-order ones (10.4 waves of 768-column rows: trace 50.5 -> 51.0 ms, replay + quantisation
+        // 51.1 -> 55.3 ms; 5.1 waves of 704-column rows 39.5 -> 40.5 and 42.5 -> 48.9 ms; 3.4 waves of 1408-column rows
+        // gain, 79.9 -> 70.9 ms, 5.7 waves of 1152-column rows do not).
+        const bool want_split = a.row_count > blocks && a.row_count % blocks != 0 && (p.per_sm == 1 || a.row_count < 3 * blocks) &&
                                 a.nm_prune == 0 && !bc && !(a.opts.flags & OBC_ENGINE_WHOLE_WAVES);
         const size_t tri = round_up((size_t)blocks * (want_split ? 2 : 1) * a.d * a.cap * sizeof(float), 256);
         const size_t gpan = p.g_vectors ? round_up((size_t)blocks * p.g_vectors * p.g_ld * sizeof(float), 256) : 0;
