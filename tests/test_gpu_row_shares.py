@@ -26,15 +26,18 @@ def _sm_count():
     return torch.cuda.get_device_properties(0).multi_processor_count
 
 
-@pytest.mark.parametrize("threads,d,extra", [(128, 300, 37), (256, 520, 11), (512, 520, 29), (0, 640, 5), (512, 1100, 3)])
-def test_row_shares_prune_trace_quant_replay(threads, d, extra):
+@pytest.mark.parametrize("threads,d,extra,waves", [(128, 300, 37, 1), (256, 520, 11, 1), (512, 520, 29, 1), (0, 640, 5, 1),
+                                                   (512, 1100, 3, 1), (512, 520, 61, 4), (256, 400, 100, 2)])
+def test_row_shares_prune_trace_quant_replay(threads, d, extra, waves):
     import paper_2208_11580_b200 as m
     m.load_library()
     m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, 0)
     plan = m.obc_engine_plan(d, True, 0)
     grid = plan["rows_per_sm"] * plan["sm_count"]
     assert d > plan["on_chip_below"]
-    rows = grid + extra                                   # one whole wave and a little: almost every block shares a row
+    # whole waves and a little: almost every block shares a row (with one row per SM shares are taken at any number of
+    # waves, otherwise up to three)
+    rows = waves * grid + extra
     W, X = obc_synth.make_small(rows, d, 3 * d + 64, 5100 + d, "relu")
     H = oracle.hessian(X).astype(np.float32)
     ld = (d + 3) // 4 * 4
