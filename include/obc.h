@@ -192,10 +192,11 @@ obc_status obc_prune_nm(const float *W, int ldw, int d_row, int d_col, int row_b
  * remaining block P with the smallest w_P^T ((Hinv)_P)^-1 w_P (ties: lowest block), compensates the other weights by
  * -Hinv[:,P] ((Hinv)_P)^-1 w_P and eliminates the members of P from the row's inverse Hessian one after the other
  * (Lemma 1) -- which is the same as eliminating the members singly in ascending order, and that is how it runs.
- *   block = 4 (the only size built); d_col a multiple of 4.  Full trace (all d_col / 4 blocks).
- *   order : d_row x d_col, the members of the t-th block at [4t, 4t+4), ascending.
- *   loss  : d_row x d_col, loss[r][4t] = the block's score, loss[r][4t+1..4t+3] = 0, so that
- *           obc_select_global_mask with k a multiple of 4 takes whole blocks, and obc_prune_apply works unchanged.
+ *   block = c = 4 or 8 (the sizes the section names; others: OBC_ERR_UNSUPPORTED); d_col a multiple of c.  Full trace
+ *           (all d_col / c blocks).
+ *   order : d_row x d_col, the members of the t-th block at [ct, ct+c), ascending.
+ *   loss  : d_row x d_col, loss[r][ct] = the block's score, loss[r][ct+1..ct+c-1] = 0, so that
+ *           obc_select_global_mask with k a multiple of c takes whole blocks, and obc_prune_apply works unchanged.
  *   w_trace: as in obc_prune_trace (one row per single elimination), nullable.
  * Always runs on the BLOCKED engine.  Workspace: obc_workspace_bytes(OBC_OP_PRUNE_BLOCKS, row_count, d_col, 0). */
 obc_status obc_prune_blocks(const float *W, int ldw, int d_row, int d_col, int row_begin, int row_count,

@@ -190,8 +190,8 @@ obc_status obc_prune_blocks(const float* W, int ldw, int d_row, int d_col, int r
     if (!engine_opts_ok(opts, &eo)) return OBC_ERR_INVALID_ARG;
     if (!rows_ok(d_row, d_col, row_begin, row_count) || !mat_ok(W, ldw, d_col) || !mat_ok(Hinv, ldhi, d_col))
         return OBC_ERR_INVALID_ARG;
-    if (!order || !loss || !row_status || d_col % 4 != 0) return OBC_ERR_INVALID_ARG;
-    if (block != 4 || d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
+    if (!order || !loss || !row_status || block <= 0 || d_col % block != 0) return OBC_ERR_INVALID_ARG;
+    if ((block != 4 && block != 8) || d_col > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     if (!mat_aligned(W, ldw) || !mat_aligned(Hinv, ldhi)) return OBC_ERR_ALIGNMENT;
     return engine_prune_blocks(W, ldw, d_row, d_col, row_begin, row_count, Hinv, ldhi, block, order, loss, w_trace,
                                row_status, ws, ws_bytes, eo, (cudaStream_t)stream);

@@ -54,10 +54,10 @@ constexpr int BLK_GS = 4;                     // forced eliminations taken toget
 
 // Per-row state in shared memory: wd, dg (FP64), perm (int32), srcm (uint16); optional: the row in original
 // order (weight trace), one byte per block of the N:M pattern.
-// (block pruning: the 6 off-diagonal entries of every 4-slot group's 4 x 4 diagonal block, FP64)
-__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm = false, bool bc = false) {
+// (block pruning, bc = block size 4 or 8: the 6 or 28 off-diagonal entries of every block's c x c diagonal block, FP64)
+__host__ __device__ inline size_t blk_state_bytes(int cap, bool wfull, bool nm = false, int bc = 0) {
     return (size_t)20 * cap + (((size_t)2 * cap + 15) & ~(size_t)15) + (wfull ? (size_t)4 * cap : 0) +
-           (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0) + (bc ? (size_t)12 * cap : 0);
+           (nm ? (((size_t)(cap >> 1) + 15) & ~(size_t)15) : 0) + (bc == 8 ? (size_t)28 * cap : (bc ? (size_t)12 * cap : 0));
 }
 // Stride of the pending vectors for a row of m slots: = 8 (mod 32), so that the tensor-core fragments of the
 // flush (4 vectors x 8 consecutive slots per load) touch 32 different banks.
@@ -609,8 +609,38 @@ __device__ __forceinline__ double block4_score(const double* w, const double* a,
     return y0 * y0 * r0 + y1 * y1 * r1 + y2 * y2 * r2 + y3 * y3 * r3;
 }
 
+// Blocks of 8: the same score by Gaussian elimination of the members in ascending order on a copy of the 8 x 8 block
+// (diagonal a, off-diagonals o packed by rows of the upper triangle: (0,1) .. (0,7), (1,2) .. (6,7)): the sum of the
+// eight single-weight losses w_i^2 / a_ii met on the way.  Returns NaN if a pivot is not positive.
+__device__ __forceinline__ int block8_index(int i, int j) { return i * (15 - i) / 2 + (j - i - 1); }      // i < j
+__device__ __noinline__ double block8_score(const double* w, const double* a, const double* o) {
+    double m[8][8], y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        y[i] = w[i]; m[i][i] = a[i];
+#pragma unroll
+        for (int j = i + 1; j < 8; ++j) m[i][j] = o[block8_index(i, j)];
+    }
+    double sc = 0.0;
+    bool ok = true;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const double dii = m[i][i], r = 1.0 / dii;
+        ok = ok && (dii > 0.0);
+        sc += y[i] * y[i] * r;
+#pragma unroll
+        for (int j = i + 1; j < 8; ++j) {
+            const double l = m[i][j] * r;
+            y[j] -= l * y[i];
+#pragma unroll
+            for (int k = j; k < 8; ++k) m[j][k] -= l * m[i][k];
+        }
+    }
+    return ok ? sc : CUDART_NAN;
+}
+
 // Q = the kernel contains the OBQ code (modes QUANT and REPLAY_QUANT); the pruning kernels are built without it.
-// BC = 4: block pruning in blocks of 4 consecutive columns (pruning kernels only), 0: single weights.
+// BC = 4 or 8: block pruning in blocks of that many consecutive columns (pruning kernels only), 0: single weights.
 // FG = the kernel takes forced eliminations (replay of a known order) four at a time: their order is known, so the
 // four pivot columns are fetched and corrected together, the 4 x 4 block of the columns at the pivot slots is
 // broadcast, and every thread carries out the four Lemma-1 eliminations on its own slots in registers -- two
@@ -643,7 +673,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
     const int nm_lg = a.nm_lg, nm_prune = a.nm_prune;
     unsigned char* blkcnt = reinterpret_cast<unsigned char*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull));
     double* boff = reinterpret_cast<double*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm));
-    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm, BC != 0));
+    float* panel = reinterpret_cast<float*>(smem + BLK_FIXED + blk_state_bytes(cap, has_wfull, has_nm, BC));
     // tail views (step-by-step phase in shared memory) share the panel's space
     const int msr = (ms + 3) & ~3;
     float* tv = panel;
@@ -744,7 +774,15 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
             if (a.mask) a.mask[(size_t)r * d + j] = 1;
         }
         if (has_nm) for (int b = tid; b < (d >> nm_lg); b += NT) blkcnt[b] = 0;
-        if (BC) {
+        if (BC == 8) {
+            for (int e = tid; e < (d >> 3) * 28; e += NT) {
+                const int g = e / 28, k = e - g * 28;
+                int ia = 0, rest = k;
+                while (rest >= 7 - ia) { rest -= 7 - ia; ++ia; }
+                const int ib = ia + 1 + rest;
+                boff[e] = (double)a.Hinv[(size_t)(8 * g + ia) * a.ldhi + 8 * g + ib];
+            }
+        } else if (BC) {
             for (int e = tid; e < (d >> 2) * 6; e += NT) {
                 const int g = e / 6, k = e - g * 6;
                 const int ia = k < 3 ? 0 : (k < 5 ? 1 : 2), ib = k < 3 ? k + 1 : (k < 5 ? k - 1 : 3);
@@ -841,8 +879,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     if (tid < nh) {
                         const int h = hl[tid], sv = mv[tid];
                         wd[h] = wd[sv]; dg[h] = dg[sv]; perm[h] = perm[sv];
-                        if (BC && (h & 3) == 0)      // holes and movers are whole aligned groups in block mode
+                        if (BC == 4 && (h & 3) == 0)      // holes and movers are whole aligned groups in block mode
                             for (int k = 0; k < 6; ++k) boff[(h >> 2) * 6 + k] = boff[(sv >> 2) * 6 + k];
+                        if (BC == 8 && (h & 7) == 0)
+                            for (int k = 0; k < 28; ++k) boff[(h >> 3) * 28 + k] = boff[(sv >> 3) * 28 + k];
                         srcm[h] = (unsigned short)h;
                         colmask[h >> 5] = 0u;
                     }
@@ -1093,8 +1133,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
 #pragma unroll
                 for (int g = 0; g < KMAX / 4; ++g) {
                     const int jb = own_slot<NT>(4 * g);
+                    if (BC == 8 && (jb & 7) != 0) continue;      // a block of 8 is scored by the owner of its first half
                     if (jb < m0 && perm[jb] >= 0) {
-                        const double sc4 = block4_score(wd + jb, dg + jb, boff + (jb >> 2) * 6);
+                        const double sc4 = BC == 8 ? block8_score(wd + jb, dg + jb, boff + (jb >> 3) * 28)
+                                                   : block4_score(wd + jb, dg + jb, boff + (jb >> 2) * 6);
                         const int o = perm[jb];
                         if (key_less(sc4, o, bs, bo)) { bs = sc4; bo = o; cslot = jb; }
                     }
@@ -1223,13 +1265,42 @@ __global__ void __launch_bounds__(NT, 512 / NT) blocked_engine_kernel(const Engi
                     wq[0] = make_double2(wv[0], wv[1]); wq[1] = make_double2(wv[2], wv[3]);
                     dq[0] = make_double2(dv[0], dv[1]); dq[1] = make_double2(dv[2], dv[3]);
                     *reinterpret_cast<float4*>(zb + jb) = make_float4(zv[0], zv[1], zv[2], zv[3]);
-                    if (BC && ((live >> (4 * g)) & 0xFu) == 0xFu && jb != (p & ~3)) {
+                    if (BC == 4 && ((live >> (4 * g)) & 0xFu) == 0xFu && jb != (p & ~3)) {
                         // Lemma 1 on the group's own 4 x 4 diagonal block (off-diagonal part; dg holds the diagonal)
                         double* o = boff + (jb >> 2) * 6;
                         const double v0 = (double)(c[4 * g] - corr[4 * g]), v1 = (double)(c[4 * g + 1] - corr[4 * g + 1]);
                         const double v2 = (double)(c[4 * g + 2] - corr[4 * g + 2]), v3 = (double)(c[4 * g + 3] - corr[4 * g + 3]);
                         o[0] -= v0 * v1 * idpp; o[1] -= v0 * v2 * idpp; o[2] -= v0 * v3 * idpp;
                         o[3] -= v1 * v2 * idpp; o[4] -= v1 * v3 * idpp; o[5] -= v2 * v3 * idpp;
+                    }
+                }
+                if (BC == 8) {
+                    // Lemma 1 on the 8 x 8 diagonal block of every other whole block: its two halves belong to
+                    // neighbouring lanes, which exchange their four column entries; the lane of the first half takes
+                    // the pairs whose smaller index is 0 or 1, the other lane the rest
+#pragma unroll
+                    for (int g = 0; g < KMAX / 4; ++g) {
+                        const int jb = own_slot<NT>(4 * g);
+                        float mine[4], other[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) mine[q] = c[4 * g + q] - corr[4 * g + q];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) other[q] = __shfl_xor_sync(0xffffffffu, mine[q], 1);
+                        if (jb < m0 && ((live >> (4 * g)) & 0xFu) == 0xFu && (jb & ~7) != (p & ~7)) {
+                            const bool first = (jb & 7) == 0;
+                            double v[8];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                v[q] = (double)(first ? mine[q] : other[q]);
+                                v[4 + q] = (double)(first ? other[q] : mine[q]);
+                            }
+                            double* o = boff + (jb >> 3) * 28;
+#pragma unroll
+                            for (int i = 0; i < 7; ++i)
+#pragma unroll
+                                for (int j = i + 1; j < 8; ++j)
+                                    if ((i < 2) == first) o[block8_index(i, j)] -= v[i] * v[j] * idpp;
+                        }
                     }
                 }
                 sa_valid = est_next;
@@ -1354,7 +1425,7 @@ static int blk_pick_ms(int d, size_t panel_bytes) {
 // Threads per block and blocks per SM by row length: short rows are bound by the latency of a step, so
 // several of them share an SM; long rows need the shared memory for pending vectors.
 // row_count = rows of the launch (0 = many).
-static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, bool bc = false,
+static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool nm = false, int bc = 0,
                      int row_count = 0, int threads = 0) {
     const int cap = (d + 3) & ~3;
     int nt = threads;
@@ -1377,7 +1448,8 @@ static bool blk_plan(int d, bool wfull, const DeviceInfo& di, BlkPlan* out, bool
     if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
     const size_t fixed = BLK_FIXED + blk_state_bytes(cap, wfull, nm, bc);
     const size_t min_panel = (size_t)4 * blk_ldz(cap);
-    while (p.per_sm > 1 && share < fixed + 4 * min_panel) {     // too little room: fewer, larger blocks
+    const size_t min_vectors = bc > 4 ? (size_t)bc : 4;         // (block pruning flushes whole blocks of bc updates)
+    while (p.per_sm > 1 && share < fixed + min_vectors * min_panel) {     // too little room: fewer, larger blocks
         p.per_sm >>= 1;
         share = (sm_total / p.per_sm - 1024) & ~(size_t)127;
         if (share > (size_t)di.smem_optin) share = (size_t)di.smem_optin;
@@ -1489,6 +1561,7 @@ static obc_status blk_launch_q(const EngineArgs& a, int blocks, size_t smem, int
 template <int NT, int KMAX>
 static obc_status blk_launch(const EngineArgs& a, int blocks, size_t smem, int sm_count, cudaStream_t stream) {
     if (a.block_c == 4) return blk_launch_q<NT, KMAX, false, 4, false>(a, blocks, smem, sm_count, stream);
+    if (a.block_c == 8) return blk_launch_q<NT, KMAX, false, 8, false>(a, blocks, smem, sm_count, stream);
     switch (a.mode) {                       // the replay modes are the ones with forced eliminations
         case MODE_QUANT:        return blk_launch_q<NT, KMAX, true, 0, false>(a, blocks, smem, sm_count, stream);
         // (with 512 threads the OBQ kernel has no registers to spare for the four columns: single steps there)
@@ -1506,17 +1579,17 @@ obc_status blocked_engine_launch(EngineArgs a, void* ws, size_t ws_bytes, cudaSt
     a.cap = (a.d + 3) & ~3;
     if (a.d > OBC_MAX_DCOL) return OBC_ERR_UNSUPPORTED;
     BlkPlan p;
-    const bool bc = a.block_c == 4;
+    const int bc = (a.block_c == 4 || a.block_c == 8) ? a.block_c : 0;      // block pruning: the block size
     if (!blk_plan(a.d, a.w_trace != nullptr, di, &p, a.nm_prune > 0, bc, a.row_count, a.opts.threads)) return OBC_ERR_UNSUPPORTED;
     a.ms = p.ms;
     a.panel_floats = p.panel_floats;
     const int mp = a.opts.max_pending;
     a.max_pending = (mp >= 1 && mp <= BLK_MAXB) ? mp : BLK_MAXB;
     if (bc) {
-        // groups of 4 slots must stay together: no on-chip tail (it compacts slot by slot), whole blocks per flush
+        // the slots of a block must stay together: no on-chip tail (it compacts slot by slot), whole blocks per flush
         a.ms = 0;
-        if (a.max_pending < 4) a.max_pending = 4;
-        if (p.panel_floats / blk_ldz(a.cap) + p.g_vectors < 4) return OBC_ERR_UNSUPPORTED;
+        if (a.max_pending < bc) a.max_pending = bc;
+        if (p.panel_floats / blk_ldz(a.cap) + p.g_vectors < bc) return OBC_ERR_UNSUPPORTED;
     }
     int blocks = di.sm_count * p.per_sm;
     if (a.row_count < blocks) blocks = a.row_count;

@@ -78,28 +78,29 @@ def test_nm_long_rows(layer):
     check_rows(Hh, W[:rows], o, loss.cpu().numpy(), gpu_w=wo, steps=steps, nm=(2, 4))
 
 
-def test_blocks_long_rows(layer):
+@pytest.mark.parametrize("c", [4, 8])
+def test_blocks_long_rows(layer, c):
     m, W, Wd, Hinv, Hh = layer
-    rows, nblk = 3, D // 8                    # compared: the first half of the blocks (the passes with vectors in global memory)
+    rows, nblk = 3, D // (2 * c)              # compared: the first half of the blocks (the passes with vectors in global memory)
     order = torch.full((rows, D), -7, dtype=torch.int32, device="cuda")
     loss = torch.full((rows, D), -7.0, dtype=torch.float32, device="cuda")
     rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
     trace = torch.zeros(rows, D + 1, D, dtype=torch.float32, device="cuda")
-    m.obc_prune_blocks(Wd[:rows], Hinv, order, loss, rs, w_trace=trace)
+    m.obc_prune_blocks(Wd[:rows], Hinv, order, loss, rs, block=c, w_trace=trace)
     torch.cuda.synchronize()
     assert int(rs.abs().sum()) == 0
     full = order.cpu().numpy()
-    assert all(sorted((full[r, ::4] // 4).tolist()) == list(range(D // 4)) for r in range(rows))
+    assert all(sorted((full[r, ::c] // c).tolist()) == list(range(D // c)) for r in range(rows))
     assert np.all(trace[:, -1].cpu().numpy() == 0.0)
-    o, l = full[:, :4 * nblk], loss.cpu().numpy().astype(np.float64)[:, :4 * nblk]
-    blocks = o[:, ::4] // 4
-    assert np.array_equal(o, (blocks[:, :, None] * 4 + np.arange(4)).reshape(rows, 4 * nblk))
-    res = oracle.run_rows_blocks(Hh.astype(np.float64), W[:rows], 4, steps=nblk, forced_blocks=blocks)
+    o, l = full[:, :c * nblk], loss.cpu().numpy().astype(np.float64)[:, :c * nblk]
+    blocks = o[:, ::c] // c
+    assert np.array_equal(o, (blocks[:, :, None] * c + np.arange(c)).reshape(rows, c * nblk))
+    res = oracle.run_rows_blocks(Hh.astype(np.float64), W[:rows], c, steps=nblk, forced_blocks=blocks)
     assert np.all(res["status"] == 0)
     differ = res["best_block"] != blocks
     assert not (differ & (res["forced_gap"] > 1e-6)).any()
-    L = res["loss"][:, ::4]
+    L = res["loss"][:, ::c]
     floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
-    assert (np.abs(l[:, ::4] - L) / (np.abs(L) + floor)).max() <= REL_TOL
+    assert (np.abs(l[:, ::c] - L) / (np.abs(L) + floor)).max() <= REL_TOL
     wscale = np.abs(W[:rows]).max(axis=1, keepdims=True)
-    assert (np.abs(trace[:, 4 * nblk].cpu().numpy() - res["w"]) / wscale).max() <= REL_TOL
+    assert (np.abs(trace[:, c * nblk].cpu().numpy() - res["w"]) / wscale).max() <= REL_TOL

@@ -468,15 +468,17 @@ def test_prune_nm_against_oracle(nm, d, rows, threads, max_pending):
     check_rows(Hinv.cpu().numpy(), W, o, loss.cpu().numpy(), gpu_w=wo, steps=steps, nm=nm)
 
 
+@pytest.mark.parametrize("c", [4, 8])
 @pytest.mark.parametrize("threads,max_pending", [(0, 0), (128, 4), (256, 9), (512, 64)])
 @pytest.mark.parametrize("d,rows,kind", [(8, 3, "correlated"), (64, 4, "relu"), (300, 4, "correlated"), (640, 3, "relu")])
-def test_prune_blocks_against_oracle(d, rows, kind, threads, max_pending):
-    """block pruning in blocks of 4 (Section 3, "Block-Sparsity", Eq. 5): block picks (margin-gated), block losses,
-    weights after a given number of blocks, and whole-block global masks"""
+def test_prune_blocks_against_oracle(d, rows, kind, threads, max_pending, c):
+    """block pruning in blocks of c = 4 or 8 (Section 3, "Block-Sparsity", Eq. 5): block picks (margin-gated), block
+    losses, weights after a given number of blocks, and whole-block global masks"""
     import paper_2208_11580_b200 as m
     m.load_library()
     m = WithEngineOpts(m, m.ENGINE_BLOCKED, threads, max_pending)
-    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1500 + d, kind)
+    d += -d % c
+    W, X = obc_synth.make_small(rows, d, 3 * d + 64, 1500 + d + c, kind)
     H = oracle.hessian(X).astype(np.float32)
     Hinv, info = m.obc_hessian_inverse(dev(H), DAMP)
     Wd = dev(W)
@@ -484,39 +486,39 @@ def test_prune_blocks_against_oracle(d, rows, kind, threads, max_pending):
     loss = torch.full((rows, d), -7.0, dtype=torch.float32, device="cuda")
     rs = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
     trace = torch.zeros(rows, d + 1, d, dtype=torch.float32, device="cuda")
-    m.obc_prune_blocks(Wd, Hinv, order, loss, rs, w_trace=trace)
+    m.obc_prune_blocks(Wd, Hinv, order, loss, rs, block=c, w_trace=trace)
     torch.cuda.synchronize()
     assert int(rs.abs().sum()) == 0
     o, l = order.cpu().numpy(), loss.cpu().numpy().astype(np.float64)
-    blocks = o[:, ::4] // 4
-    assert np.array_equal(o, (blocks[:, :, None] * 4 + np.arange(4)).reshape(rows, d))        # members ascending
-    assert all(sorted(blocks[r].tolist()) == list(range(d // 4)) for r in range(rows))
-    assert np.all(l.reshape(rows, d // 4, 4)[:, :, 1:] == 0.0)
+    blocks = o[:, ::c] // c
+    assert np.array_equal(o, (blocks[:, :, None] * c + np.arange(c)).reshape(rows, d))        # members ascending
+    assert all(sorted(blocks[r].tolist()) == list(range(d // c)) for r in range(rows))
+    assert np.all(l.reshape(rows, d // c, c)[:, :, 1:] == 0.0)
     Hh = Hinv.cpu().numpy().astype(np.float64)
-    res = oracle.run_rows_blocks(Hh, W, 4, forced_blocks=blocks)
+    res = oracle.run_rows_blocks(Hh, W, c, forced_blocks=blocks)
     assert np.all(res["status"] == 0)
     differ = res["best_block"] != blocks
     assert not (differ & (res["forced_gap"] > 1e-6)).any()
-    L = res["loss"][:, ::4]
+    L = res["loss"][:, ::c]
     floor = 1e-7 * np.abs(L).max(axis=1, keepdims=True)
-    assert (np.abs(l[:, ::4] - L) / (np.abs(L) + floor)).max() <= REL_TOL
+    assert (np.abs(l[:, ::c] - L) / (np.abs(L) + floor)).max() <= REL_TOL
     assert np.all(trace[:, -1].cpu().numpy() == 0.0)
-    # weights after nb blocks (trace row 4*nb) against the oracle stopped there
+    # weights after nb blocks (trace row c*nb) against the oracle stopped there
     wscale = np.abs(W).max(axis=1, keepdims=True)
-    for nb in (1, d // 8, d // 4 - 1):
-        part = oracle.run_rows_blocks(Hh, W, 4, steps=nb, forced_blocks=blocks[:, :nb])
-        assert (np.abs(trace[:, 4 * nb].cpu().numpy() - part["w"]) / wscale).max() <= REL_TOL
-    # global step on whole blocks: k a multiple of 4
-    k = (rows * d // 8) * 4
+    for nb in sorted({1, max(1, d // (2 * c)), max(1, d // c - 1)}):
+        part = oracle.run_rows_blocks(Hh, W, c, steps=nb, forced_blocks=blocks[:, :nb])
+        assert (np.abs(trace[:, c * nb].cpu().numpy() - part["w"]) / wscale).max() <= REL_TOL
+    # global step on whole blocks: k a multiple of c
+    k = (rows * d // (2 * c)) * c
     counts = torch.zeros(rows, dtype=torch.int32, device="cuda")
     mask = torch.zeros(rows, d, dtype=torch.uint8, device="cuda")
     m.obc_select_global_mask(loss, order, k, counts, mask)
-    c, mk = counts.cpu().numpy(), mask.cpu().numpy()
-    assert np.all(c % 4 == 0) and int((mk == 0).sum()) == k
-    per_block = mk.reshape(rows, d // 4, 4).sum(axis=2)
-    assert np.all((per_block == 0) | (per_block == 4))
+    cn, mk = counts.cpu().numpy(), mask.cpu().numpy()
+    assert np.all(cn % c == 0) and int((mk == 0).sum()) == k
+    per_block = mk.reshape(rows, d // c, c).sum(axis=2)
+    assert np.all((per_block == 0) | (per_block == c))
     oc, om = oracle.global_mask(l, o, k)
-    assert np.array_equal(c, oc) and np.array_equal(mk, om)
+    assert np.array_equal(cn, oc) and np.array_equal(mk, om)
 
 
 def test_prune_trace_at_maximum_row_length(obc):

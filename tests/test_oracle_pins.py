@@ -360,13 +360,13 @@ def test_pin_nm_pattern(nm):
         assert np.array_equal(ro["order"][r], np.array(sorted(want, key=lambda j: (score[r, j], j))))
 
 
-@pytest.mark.parametrize("c", [2, 4])
+@pytest.mark.parametrize("c", [2, 4, 8])
 def test_pin_block_pruning(c):
     """Block pruning (Section 3, "Block-Sparsity", Eq. 5): (1) every pick is the brute-force minimiser over the remaining
     blocks of the true loss increase, which is half the recorded block score; (2) after every block step the
     remaining weights are the masked least-squares optimum and the reduced inverse is inv(H[M,M]); (3) with c = 1 the
     procedure is Algorithm 1; (4) with a diagonal Hessian the block score is sum w_j^2 H_jj over the block."""
-    d = 12
+    d = 12 if c < 8 else 24
     W, X, Hd, Hinv, X_aug = _problem(3, d, 70, 41 + c)
     nblk = d // c
     for r in range(W.shape[0]):
